@@ -1,0 +1,177 @@
+/*
+ * tq.h -- C ABI of libtq: truncated quantization of heavy-tailed gradients on one GPU.
+ *
+ * The library implements the per-round hot path of Algorithm 1 (TQSGD) of "Improved
+ * Quantization Strategies for Managing Heavy-tailed Gradients in Distributed Learning":
+ *
+ *   client i :  statistics of g_i  ->  (alpha, codebook)            tq_stats, tq_params
+ *               Q_lambda[T_alpha(g_i)], b bits per element, packed   tq_compress
+ *   server   :  mean over the N clients of the dequantized codes     tq_decompress_aggregate
+ *
+ * The N clients ("workers") are N gradient slices resident on one GPU.
+ *
+ * Conventions
+ *   - "dev" pointers are CUDA device pointers owned by the caller; "host" pointers are ordinary
+ *     host memory.  The library allocates no device memory and frees nothing.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  The four compute
+ *     calls only enqueue work on it; none of them synchronises.
+ *   - num_levels L = 2^bits is the number of quantization points; the paper's s = 2^b - 1 is the
+ *     number of intervals, s = L - 1 (Section 3.1).  bits is 1, 2, 3 or 4.
+ *   - Every call returns a tq_status; nothing throws or aborts, kernels never trap.
+ *   - NaN gradients are counted by tq_stats and quantized as -alpha (code 0); +-Inf as +-alpha.
+ *
+ * Arithmetic that decides a code is fp32 with one rounding per operation (no contraction), and the
+ * random bits are a pure function of (seed, worker, element index), so a packed buffer is a
+ * deterministic function of its inputs.
+ */
+#ifndef TQ_H_
+#define TQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define TQ_MAX_LEVELS 16
+#define TQ_MAX_WORKERS 64
+
+typedef enum {
+    TQ_OK = 0,
+    TQ_ERR_INVALID_ARG = -1,       /* null pointer, bad enum, N out of range, bits mismatch */
+    TQ_ERR_DOMAIN = -2,            /* gamma <= 2, rho outside (0, 0.5), g_min <= 0, alpha <= 0 */
+    TQ_ERR_ALIGNMENT = -3,         /* a device pointer or stride misses its stated alignment */
+    TQ_ERR_BUFFER_TOO_SMALL = -4,  /* packed stride or workspace smaller than required */
+    TQ_ERR_DEGENERATE_LEVELS = -5, /* codebook not strictly increasing in fp32 */
+    TQ_ERR_CUDA = -6               /* a CUDA runtime call failed; see tq_last_cuda_error */
+} tq_status;
+
+typedef enum { TQ_F32 = 0, TQ_BF16 = 1 } tq_dtype;               /* gradient storage type */
+typedef enum { TQ_UNIFORM = 0, TQ_NONUNIFORM = 1 } tq_mode;
+typedef enum {
+    TQ_ALPHA_CLOSED = 0,       /* alpha' : the boxed equation with Q = 1 (text after Theorem 1) */
+    TQ_ALPHA_FIXED_POINT = 1,  /* iterate the boxed equation of Section 4.1 / 4.2 */
+    TQ_ALPHA_USER = 2          /* caller supplies alpha */
+} tq_alpha_rule;
+
+enum { TQ_FLAG_ALPHA_CAPPED = 1, TQ_FLAG_ALPHA_AT_GMIN = 2, TQ_FLAG_GAMMA_FROM_MLE = 4 };
+
+/* Statistics of one worker's gradient; 64 bytes, written on the device by tq_stats. */
+typedef struct {
+    uint64_t d;             /* elements seen */
+    uint64_t n_tail;        /* #{ j : |g_j| > g_min }, both signs pooled */
+    uint64_t n_nonfinite;   /* NaN / Inf elements, excluded from every sum */
+    double sum_abs;         /* sum |g_j| */
+    double sum_sq;          /* sum g_j^2 */
+    double sum_log_tail;    /* sum over the tail of ln(|g_j| / g_min) */
+    float max_abs;          /* max |g_j| over finite elements */
+    float g_min;            /* threshold used: the caller's, or kappa * mean|g| */
+    uint64_t reserved;
+} tq_stats_t;
+
+/* Quantizer of one worker; plain data, produced on the host, passed to the kernels by value. */
+typedef struct {
+    uint32_t bits;          /* b */
+    uint32_t num_levels;    /* L = 2^b */
+    uint32_t mode;          /* tq_mode */
+    uint32_t flags;         /* TQ_FLAG_* */
+    float alpha;            /* truncation threshold, = levels[L-1] */
+    float inv_step;         /* uniform mode: (L-1) / (2 alpha), rounded up */
+    float gamma;            /* tail exponent used */
+    float g_min;
+    float rho;              /* one-sided tail mass n_tail / (2 d) */
+    int32_t iterations;     /* fixed-point iterations spent on alpha */
+    float reserved[2];
+    float levels[TQ_MAX_LEVELS];     /* l_0 = -alpha < ... < l_{L-1} = alpha */
+    float inv_width[TQ_MAX_LEVELS];  /* 1 / (l_{k+1} - l_k), rounded up, k < L-1 */
+} tq_params_t;
+
+/* Words (uint32) of one worker's packed buffer: ceil(d * bits / 32) rounded up to a multiple of 4.
+ * Wire format (the paper only says "b bits per element", Section 2): code j occupies bits
+ * [j*bits, (j+1)*bits) of an LSB-first stream over little-endian 32-bit words; unused bits are 0. */
+size_t tq_packed_words(uint64_t d, uint32_t bits);
+
+/* Bytes of device scratch tq_stats needs for n_workers slices (block partials + tickets). */
+size_t tq_stats_workspace_bytes(uint32_t n_workers);
+
+/*
+ * Statistics reduction (Section 5: gamma = 1 + n [sum ln(g_j / g_min)]^-1 over g_j > g_min;
+ * Section 4.1: rho = tail mass beyond g_min).  One 64-byte record per worker.
+ *   grad_dev     [n_workers][grad_stride] elements of `dtype`, 32-byte aligned; worker i's slice is
+ *                the first d elements of row i.  grad_stride (elements) must keep rows 32-byte aligned.
+ *   g_min        > 0: threshold for the tail.  <= 0: each worker uses kappa * mean|g| of its own
+ *                slice (one extra pass over the data).
+ *   stats_dev    [n_workers] tq_stats_t, device memory, 8-byte aligned; valid when the stream reaches
+ *                the end of this call's work (copy it back to the host for tq_params).
+ *   workspace_dev, ws_bytes   device scratch of at least tq_stats_workspace_bytes(n_workers), 256-byte
+ *                aligned; contents need not be initialised and are not meaningful afterwards.  Calls
+ *                sharing one workspace must not overlap on the device.
+ * Sums are accumulated in fp32 over runs of 16 elements and in fp64 beyond; counts and max are exact.
+ * d = 0 is allowed (all-zero records).  Errors: INVALID_ARG, ALIGNMENT, BUFFER_TOO_SMALL, CUDA.
+ */
+tq_status tq_stats(const void* grad_dev, tq_dtype dtype, uint64_t d, uint64_t grad_stride,
+                   uint32_t n_workers, float g_min, float kappa, tq_stats_t* stats_dev,
+                   void* workspace_dev, size_t ws_bytes, void* stream);
+
+/*
+ * Parameter design on the host (Section 4), O(L) work in double precision.
+ *   stats_host   one record copied back from tq_stats.
+ *   gamma        tail exponent of the power-law model; NaN = use the maximum-likelihood estimate.
+ *                Must exceed 2.
+ *   alpha_rule   CLOSED: alpha' = g_min [2 rho s^2 / (gamma-2)]^(1/(gamma-1)).
+ *                FIXED_POINT: the boxed equations alpha = g_min [2 rho s^2 / ((gamma-2) Q(alpha))]^(1/(gamma-1))
+ *                with Q = Q_U (uniform, Section 4.1) or Q_N (non-uniform, Section 4.2), evaluated on
+ *                the model density (flat below g_min, power law above), iterated from alpha' until the
+ *                relative change is <= 1e-12 or 10000 iterations.  Both are clamped to
+ *                [g_min, max_abs] (flags ALPHA_AT_GMIN / ALPHA_CAPPED).
+ *                USER: alpha_user, unclamped.
+ *   mode         UNIFORM: l_k = -alpha + k 2 alpha / s.  NONUNIFORM: the boxed density
+ *                lambda_s proportional to p^(1/3) (Section 4.2), turned into levels by
+ *                integral_{-alpha}^{l_k} lambda_s = k.
+ * Errors: INVALID_ARG, DOMAIN, DEGENERATE_LEVELS.  out_host is unspecified on error.
+ */
+tq_status tq_params(const tq_stats_t* stats_host, uint32_t num_levels, tq_mode mode, double gamma,
+                    tq_alpha_rule alpha_rule, double alpha_user, tq_params_t* out_host);
+
+/* Quantizer for a caller-supplied codebook (any strictly increasing levels with
+ * levels[0] = -levels[L-1]; Section 3.1's general codebook).  Fills inv_width / inv_step. */
+tq_status tq_params_from_levels(const float* levels_host, uint32_t num_levels, tq_mode mode,
+                                tq_params_t* out_host);
+
+/*
+ * Client side: truncate (Section 3.1, truncation equation), stochastically round onto the codebook
+ * (quantizer equation) and pack, for n_workers slices in one launch.
+ *   grad_dev     as for tq_stats.
+ *   params_host  [n_workers]; all must have the same bits.  Copied during the call.
+ *   seed, first_worker   element j of slice i draws its 16 random bits from Philox4x32-10 with
+ *                key = seed and counter = (j >> 3, first_worker + i, 0), slot j & 7.
+ *   packed_dev   [n_workers][words_stride] uint32, 16-byte aligned, words_stride a multiple of 4 and
+ *                >= tq_packed_words(d, bits).  The first tq_packed_words(d, bits) words of each row
+ *                are written (padding as zeros); words beyond are untouched.
+ * Decision per element: t = clip(g); interval k and p = (t - l_k) / (l_{k+1} - l_k) in fp32;
+ * T = rint(p * 2^16); code = k + [r < T].  Errors: INVALID_ARG, ALIGNMENT, BUFFER_TOO_SMALL, CUDA.
+ */
+tq_status tq_compress(const void* grad_dev, tq_dtype dtype, uint64_t d, uint64_t grad_stride,
+                      uint32_t n_workers, const tq_params_t* params_host, uint64_t seed,
+                      uint32_t first_worker, uint32_t* packed_dev, size_t words_stride, void* stream);
+
+/*
+ * Server side (Algorithm 1, aggregation step): out_j = sum_i w_i * levels_i[code_ij].
+ *   weights_host NULL: w_i = 1/N (Lemma 2): fp32 adds in worker order, then one division by N.
+ *                else [n_workers] fp32: each product is rounded, then added in worker order.
+ *   out_dev      [d] fp32, 16-byte aligned.
+ * Errors: INVALID_ARG, ALIGNMENT, BUFFER_TOO_SMALL, CUDA.
+ */
+tq_status tq_decompress_aggregate(const uint32_t* packed_dev, size_t words_stride, uint32_t n_workers,
+                                  uint64_t d, const tq_params_t* params_host, const float* weights_host,
+                                  float* out_dev, void* stream);
+
+const char* tq_strerror(tq_status status);
+int tq_last_cuda_error(void);   /* cudaError_t of the last failed runtime call on this thread, else 0 */
+uint64_t tq_kernel_launches(void); /* kernels launched by this library in this process so far */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TQ_H_ */

@@ -99,6 +99,8 @@ def lib() -> C.CDLL:
         L.orc_decision.restype = None
         L.orc_quantize.argtypes = [C.c_void_p, u64, P(Params), u64, u32, C.c_void_p]
         L.orc_quantize.restype = None
+        L.orc_quantize_window.argtypes = [C.c_void_p, u64, u64, P(Params), u64, u32, C.c_void_p]
+        L.orc_quantize_window.restype = None
         L.orc_packed_words.argtypes = [u64, u32]; L.orc_packed_words.restype = u64
         L.orc_pack.argtypes = [C.c_void_p, u64, u32, C.c_void_p, u64]; L.orc_pack.restype = None
         L.orc_unpack.argtypes = [C.c_void_p, u64, u32, C.c_void_p]; L.orc_unpack.restype = None
@@ -216,6 +218,14 @@ def quantize(g: np.ndarray, p: Params, seed: int, worker: int) -> np.ndarray:
     g = _f32(g)
     codes = np.empty(g.size, dtype=np.uint8)
     lib().orc_quantize(g.ctypes.data, g.size, C.byref(p), seed, worker, codes.ctypes.data)
+    return codes
+
+
+def quantize_window(g: np.ndarray, j0: int, p: Params, seed: int, worker: int) -> np.ndarray:
+    """Codes of elements j0 .. j0+len(g)-1 of a longer vector (``g`` holds just that window)."""
+    g = _f32(g)
+    codes = np.empty(g.size, dtype=np.uint8)
+    lib().orc_quantize_window(g.ctypes.data, g.size, j0, C.byref(p), seed, worker, codes.ctypes.data)
     return codes
 
 

@@ -458,6 +458,15 @@ void orc_quantize(const float *g, uint64_t d, const orc_params_t *q, uint64_t se
         codes[j] = (uint8_t)orc_code_at(q, g[j], seed, worker, j);
 }
 
+/* Codes of the n elements j0 .. j0+n-1 of a longer vector (g points at element j0): the random
+ * bits depend on the absolute index, so a window of a large gradient can be checked on its own. */
+void orc_quantize_window(const float *g, uint64_t n, uint64_t j0, const orc_params_t *q, uint64_t seed,
+                         uint32_t worker, uint8_t *codes)
+{
+    for (uint64_t i = 0; i < n; ++i)
+        codes[i] = (uint8_t)orc_code_at(q, g[i], seed, worker, j0 + i);
+}
+
 /* R12: words needed for d codes of `bits` bits, rounded up to a multiple of 4 words. */
 uint64_t orc_packed_words(uint64_t d, uint32_t bits)
 {

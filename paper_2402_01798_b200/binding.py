@@ -1,0 +1,201 @@
+"""ctypes binding of libtq.so: same names and argument order as include/tq.h.
+
+Only argument marshalling happens here.  Tensors are torch tensors used as typed device
+buffers; the stream is torch's current CUDA stream unless one is given.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import math
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libtq.so")
+
+MAX_LEVELS, MAX_WORKERS = 16, 64
+OK, ERR_INVALID_ARG, ERR_DOMAIN, ERR_ALIGNMENT, ERR_BUFFER_TOO_SMALL, ERR_DEGENERATE_LEVELS, ERR_CUDA = \
+    0, -1, -2, -3, -4, -5, -6
+F32, BF16 = 0, 1
+UNIFORM, NONUNIFORM = 0, 1
+ALPHA_CLOSED, ALPHA_FIXED_POINT, ALPHA_USER = 0, 1, 2
+FLAG_ALPHA_CAPPED, FLAG_ALPHA_AT_GMIN, FLAG_GAMMA_FROM_MLE = 1, 2, 4
+
+EXPORTS = ("tq_packed_words", "tq_stats_workspace_bytes", "tq_stats", "tq_params", "tq_params_from_levels",
+           "tq_compress", "tq_decompress_aggregate", "tq_strerror", "tq_last_cuda_error", "tq_kernel_launches")
+
+
+class Stats(C.Structure):
+    """tq_stats_t (64 bytes)."""
+    _fields_ = [("d", C.c_uint64), ("n_tail", C.c_uint64), ("n_nonfinite", C.c_uint64),
+                ("sum_abs", C.c_double), ("sum_sq", C.c_double), ("sum_log_tail", C.c_double),
+                ("max_abs", C.c_float), ("g_min", C.c_float), ("reserved", C.c_uint64)]
+
+
+class Params(C.Structure):
+    """tq_params_t (176 bytes)."""
+    _fields_ = [("bits", C.c_uint32), ("num_levels", C.c_uint32), ("mode", C.c_uint32), ("flags", C.c_uint32),
+                ("alpha", C.c_float), ("inv_step", C.c_float), ("gamma", C.c_float), ("g_min", C.c_float),
+                ("rho", C.c_float), ("iterations", C.c_int32), ("reserved", C.c_float * 2),
+                ("levels", C.c_float * MAX_LEVELS), ("inv_width", C.c_float * MAX_LEVELS)]
+
+
+assert C.sizeof(Stats) == 64 and C.sizeof(Params) == 176
+
+
+class TqError(RuntimeError):
+    def __init__(self, status: int, where: str, detail: str = ""):
+        super().__init__(f"{where}: {detail or status} (status {status})")
+        self.status = status
+
+
+_lib: Optional[C.CDLL] = None
+
+
+def lib() -> C.CDLL:
+    """Load libtq.so.  There is no fallback: a missing library is an error."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2402_01798_b200.build` "
+                "(there is no CPU or PyTorch fallback for the compressor)")
+        L = C.CDLL(LIB_PATH)
+        vp, u32, u64, f32, f64, sz = C.c_void_p, C.c_uint32, C.c_uint64, C.c_float, C.c_double, C.c_size_t
+        L.tq_packed_words.argtypes = [u64, u32]; L.tq_packed_words.restype = sz
+        L.tq_stats_workspace_bytes.argtypes = [u32]; L.tq_stats_workspace_bytes.restype = sz
+        L.tq_stats.argtypes = [vp, C.c_int, u64, u64, u32, f32, f32, vp, vp, sz, vp]; L.tq_stats.restype = C.c_int
+        L.tq_params.argtypes = [C.POINTER(Stats), u32, C.c_int, f64, C.c_int, f64, C.POINTER(Params)]
+        L.tq_params.restype = C.c_int
+        L.tq_params_from_levels.argtypes = [C.POINTER(f32), u32, C.c_int, C.POINTER(Params)]
+        L.tq_params_from_levels.restype = C.c_int
+        L.tq_compress.argtypes = [vp, C.c_int, u64, u64, u32, C.POINTER(Params), u64, u32, vp, sz, vp]
+        L.tq_compress.restype = C.c_int
+        L.tq_decompress_aggregate.argtypes = [vp, sz, u32, u64, C.POINTER(Params), C.POINTER(f32), vp, vp]
+        L.tq_decompress_aggregate.restype = C.c_int
+        L.tq_strerror.argtypes = [C.c_int]; L.tq_strerror.restype = C.c_char_p
+        L.tq_last_cuda_error.restype = C.c_int
+        L.tq_kernel_launches.restype = u64
+        _lib = L
+    return _lib
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        L = lib()
+        detail = L.tq_strerror(status).decode()
+        if status == ERR_CUDA:
+            detail += f" (cudaError {L.tq_last_cuda_error()})"
+        raise TqError(status, where, detail)
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError("gradient must be float32 or bfloat16")
+
+
+def _grad_layout(grad: torch.Tensor, d: Optional[int]):
+    """(n_workers, d, stride) of a [N, stride] or [d] gradient tensor on the GPU."""
+    if not grad.is_cuda:
+        raise ValueError("gradient must be a CUDA tensor")
+    if grad.dim() == 1:
+        grad = grad.unsqueeze(0)
+    if grad.dim() != 2 or grad.stride(1) != 1:
+        raise ValueError("gradient must be [N, stride] with unit inner stride")
+    n, width = grad.shape
+    return n, (width if d is None else d), (grad.stride(0) if n > 1 else width)
+
+
+def _params_array(params: Sequence[Params]):
+    return (Params * len(params))(*params)
+
+
+# ------------------------------------------------------------------------------------------------
+def tq_packed_words(d: int, bits: int) -> int:
+    return int(lib().tq_packed_words(d, bits))
+
+
+def tq_stats_workspace_bytes(n_workers: int) -> int:
+    return int(lib().tq_stats_workspace_bytes(n_workers))
+
+
+def tq_stats(grad: torch.Tensor, d: Optional[int] = None, g_min: float = 0.0, kappa: float = 1.0,
+             stats_dev: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None, stream=None):
+    """Enqueue the statistics reduction; returns the device tensor holding n_workers 64-byte records."""
+    n, d, stride = _grad_layout(grad, d)
+    if stats_dev is None:
+        stats_dev = torch.empty(n * 64, dtype=torch.uint8, device=grad.device)
+    if workspace is None:
+        workspace = torch.empty(tq_stats_workspace_bytes(n), dtype=torch.uint8, device=grad.device)
+    _check(lib().tq_stats(grad.data_ptr(), _dtype_code(grad), d, stride, n, g_min, kappa, stats_dev.data_ptr(),
+                          workspace.data_ptr(), workspace.numel(), _stream(stream)), "tq_stats")
+    return stats_dev
+
+
+def stats_to_host(stats_dev: torch.Tensor):
+    """Copy the records back (synchronises the current stream) and view them as Stats structures."""
+    raw = stats_dev.cpu().numpy().tobytes()
+    n = len(raw) // 64
+    return [Stats.from_buffer_copy(raw[i * 64:(i + 1) * 64]) for i in range(n)]
+
+
+def tq_params(stats: Stats, num_levels: int, mode: int, gamma: float = math.nan,
+              alpha_rule: int = ALPHA_FIXED_POINT, alpha_user: float = 0.0) -> Params:
+    p = Params()
+    _check(lib().tq_params(C.byref(stats), num_levels, mode, gamma, alpha_rule, alpha_user, C.byref(p)), "tq_params")
+    return p
+
+
+def tq_params_from_levels(levels: Sequence[float], mode: int = NONUNIFORM) -> Params:
+    arr = (C.c_float * len(levels))(*[float(x) for x in levels])
+    p = Params()
+    _check(lib().tq_params_from_levels(arr, len(levels), mode, C.byref(p)), "tq_params_from_levels")
+    return p
+
+
+def tq_compress(grad: torch.Tensor, params: Sequence[Params], seed: int, first_worker: int = 0,
+                d: Optional[int] = None, packed: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Enqueue truncate + stochastic round + pack for all rows of ``grad``; returns [N, words] int32."""
+    n, d, stride = _grad_layout(grad, d)
+    if len(params) != n:
+        raise ValueError("one Params per worker")
+    if packed is None:
+        packed = torch.empty((n, tq_packed_words(d, params[0].bits)), dtype=torch.int32, device=grad.device)
+    words_stride = packed.stride(0) if packed.dim() == 2 and n > 1 else packed.shape[-1]
+    _check(lib().tq_compress(grad.data_ptr(), _dtype_code(grad), d, stride, n, _params_array(params),
+                             seed & 0xFFFFFFFFFFFFFFFF, first_worker, packed.data_ptr(), words_stride,
+                             _stream(stream)), "tq_compress")
+    return packed
+
+
+def tq_decompress_aggregate(packed: torch.Tensor, d: int, params: Sequence[Params],
+                            weights: Optional[Sequence[float]] = None, out: Optional[torch.Tensor] = None,
+                            stream=None) -> torch.Tensor:
+    """Enqueue unpack + dequantize + average of the N packed rows; returns the [d] fp32 update."""
+    if not packed.is_cuda or packed.dim() != 2:
+        raise ValueError("packed must be a [N, words] CUDA tensor")
+    n = packed.shape[0]
+    if len(params) != n:
+        raise ValueError("one Params per worker")
+    if out is None:
+        out = torch.empty(d, dtype=torch.float32, device=packed.device)
+    w = None if weights is None else (C.c_float * n)(*[float(x) for x in weights])
+    words_stride = packed.stride(0) if n > 1 else packed.shape[1]
+    _check(lib().tq_decompress_aggregate(packed.data_ptr(), words_stride, n, d, _params_array(params), w,
+                                         out.data_ptr(), _stream(stream)), "tq_decompress_aggregate")
+    return out
+
+
+def tq_kernel_launches() -> int:
+    return int(lib().tq_kernel_launches())

@@ -1,0 +1,129 @@
+// The C ABI of libtq (declared in include/tq.h): argument checking and kernel launches.
+#include <atomic>
+#include <cstdint>
+
+#include "tq.h"
+#include "tq_launch.h"
+
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+std::atomic<uint64_t> g_launches{0};
+
+tq_status cuda_failed(cudaError_t e) {
+    g_last_cuda_error = static_cast<int>(e);
+    return TQ_ERR_CUDA;
+}
+bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+size_t elem_size(tq_dtype t) { return t == TQ_BF16 ? 2 : 4; }
+
+// common checks on a [n_workers][grad_stride] gradient block
+tq_status check_grad(const void* grad, tq_dtype dtype, uint64_t d, uint64_t stride, uint32_t n) {
+    if (dtype != TQ_F32 && dtype != TQ_BF16) return TQ_ERR_INVALID_ARG;
+    if (n == 0 || n > TQ_MAX_WORKERS) return TQ_ERR_INVALID_ARG;
+    if (d > (1ull << 40)) return TQ_ERR_INVALID_ARG;
+    if (d && !grad) return TQ_ERR_INVALID_ARG;
+    if (stride < d) return TQ_ERR_INVALID_ARG;
+    if (!aligned(grad, 32)) return TQ_ERR_ALIGNMENT;
+    if (n > 1 && (stride * elem_size(dtype)) % 32 != 0) return TQ_ERR_ALIGNMENT;
+    return TQ_OK;
+}
+
+tq_status check_params(const tq_params_t* p, uint32_t n, uint32_t* bits) {
+    if (!p) return TQ_ERR_INVALID_ARG;
+    const uint32_t b = p[0].bits;
+    if (b < 1 || b > 4) return TQ_ERR_INVALID_ARG;
+    for (uint32_t i = 0; i < n; ++i) {
+        if (p[i].bits != b || p[i].num_levels != (1u << b)) return TQ_ERR_INVALID_ARG;
+        if (p[i].mode != TQ_UNIFORM && p[i].mode != TQ_NONUNIFORM) return TQ_ERR_INVALID_ARG;
+        if (!(p[i].alpha > 0.0f)) return TQ_ERR_DOMAIN;
+    }
+    *bits = b;
+    return TQ_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t tq_packed_words(uint64_t d, uint32_t bits) {
+    const uint64_t raw = (d * bits + 31) / 32;
+    return static_cast<size_t>((raw + 3) / 4 * 4);
+}
+
+size_t tq_stats_workspace_bytes(uint32_t n_workers) { return tq::stats_workspace_bytes(n_workers); }
+
+tq_status tq_stats(const void* grad_dev, tq_dtype dtype, uint64_t d, uint64_t grad_stride, uint32_t n_workers,
+                   float g_min, float kappa, tq_stats_t* stats_dev, void* workspace_dev, size_t ws_bytes,
+                   void* stream) {
+    if (tq_status s = check_grad(grad_dev, dtype, d, grad_stride, n_workers)) return s;
+    if (!stats_dev || !workspace_dev) return TQ_ERR_INVALID_ARG;
+    if (!(g_min > 0.0f) && !(kappa > 0.0f)) return TQ_ERR_INVALID_ARG;
+    if (!aligned(stats_dev, 8) || !aligned(workspace_dev, 256)) return TQ_ERR_ALIGNMENT;
+    if (ws_bytes < tq::stats_workspace_bytes(n_workers)) return TQ_ERR_BUFFER_TOO_SMALL;
+    tq::StatsCall c{grad_dev, dtype == TQ_BF16, d, grad_stride, n_workers, g_min, kappa, stats_dev, workspace_dev,
+                    static_cast<cudaStream_t>(stream)};
+    int launched = 0;
+    const cudaError_t e = tq::launch_stats(c, &launched);
+    g_launches += static_cast<uint64_t>(launched);
+    return e == cudaSuccess ? TQ_OK : cuda_failed(e);
+}
+
+tq_status tq_compress(const void* grad_dev, tq_dtype dtype, uint64_t d, uint64_t grad_stride, uint32_t n_workers,
+                      const tq_params_t* params_host, uint64_t seed, uint32_t first_worker, uint32_t* packed_dev,
+                      size_t words_stride, void* stream) {
+    if (tq_status s = check_grad(grad_dev, dtype, d, grad_stride, n_workers)) return s;
+    uint32_t bits = 0;
+    if (tq_status s = check_params(params_host, n_workers, &bits)) return s;
+    for (uint32_t i = 1; i < n_workers; ++i)
+        if (params_host[i].mode != params_host[0].mode) return TQ_ERR_INVALID_ARG;
+    const size_t need = tq_packed_words(d, bits);
+    if (need && !packed_dev) return TQ_ERR_INVALID_ARG;
+    if (!aligned(packed_dev, 16) || words_stride % 4 != 0) return TQ_ERR_ALIGNMENT;
+    if (words_stride < need) return TQ_ERR_BUFFER_TOO_SMALL;
+    if (d == 0) return TQ_OK;
+    tq::CompressCall c{grad_dev, dtype == TQ_BF16, d, grad_stride, n_workers, params_host, bits,
+                       params_host[0].mode == TQ_NONUNIFORM, seed, first_worker, packed_dev, words_stride, need,
+                       static_cast<cudaStream_t>(stream)};
+    const cudaError_t e = tq::launch_compress(c);
+    if (e != cudaSuccess) return cuda_failed(e);
+    g_launches += 1;
+    return TQ_OK;
+}
+
+tq_status tq_decompress_aggregate(const uint32_t* packed_dev, size_t words_stride, uint32_t n_workers, uint64_t d,
+                                  const tq_params_t* params_host, const float* weights_host, float* out_dev,
+                                  void* stream) {
+    if (n_workers == 0 || n_workers > TQ_MAX_WORKERS || d > (1ull << 40)) return TQ_ERR_INVALID_ARG;
+    uint32_t bits = 0;
+    if (tq_status s = check_params(params_host, n_workers, &bits)) return s;
+    const size_t need = tq_packed_words(d, bits);
+    if (d && (!packed_dev || !out_dev)) return TQ_ERR_INVALID_ARG;
+    if (!aligned(packed_dev, 16) || words_stride % 4 != 0 || !aligned(out_dev, 32)) return TQ_ERR_ALIGNMENT;
+    if (words_stride < need) return TQ_ERR_BUFFER_TOO_SMALL;
+    if (d == 0) return TQ_OK;
+    tq::DecompressCall c{packed_dev, words_stride, need, n_workers, d, params_host, weights_host, bits, out_dev,
+                         static_cast<cudaStream_t>(stream)};
+    const cudaError_t e = tq::launch_decompress(c);
+    if (e != cudaSuccess) return cuda_failed(e);
+    g_launches += 1;
+    return TQ_OK;
+}
+
+const char* tq_strerror(tq_status s) {
+    switch (s) {
+        case TQ_OK: return "ok";
+        case TQ_ERR_INVALID_ARG: return "invalid argument";
+        case TQ_ERR_DOMAIN: return "parameter outside the model's domain";
+        case TQ_ERR_ALIGNMENT: return "pointer or stride not aligned as required";
+        case TQ_ERR_BUFFER_TOO_SMALL: return "buffer too small";
+        case TQ_ERR_DEGENERATE_LEVELS: return "codebook not strictly increasing in fp32";
+        case TQ_ERR_CUDA: return "CUDA runtime error";
+    }
+    return "unknown status";
+}
+
+int tq_last_cuda_error(void) { return g_last_cuda_error; }
+uint64_t tq_kernel_launches(void) { return g_launches.load(); }
+
+}  // extern "C"

@@ -1,0 +1,94 @@
+// Device-side building blocks shared by the libtq kernels (sm_100a).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "tq.h"
+
+namespace tq {
+
+constexpr int kThreads = 256;
+constexpr float kMagic = 8388608.0f;          // 2^23: adding it leaves an integer in the mantissa
+constexpr uint32_t kMagicBits = 0x4B000000u;  // bit pattern of 2^23
+
+// ---- 256-bit global accesses (one full 32-byte sector per lane) ---------------------------------
+__device__ __forceinline__ void ldg256_stream(const void* p, uint32_t (&v)[8]) {
+    asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                 : "l"(p));
+}
+__device__ __forceinline__ void stg256(void* p, const float (&v)[8]) {
+    asm volatile("st.global.v8.f32 [%8], {%0,%1,%2,%3,%4,%5,%6,%7};"
+                 :: "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]), "l"(p)
+                 : "memory");
+}
+
+// Eight consecutive gradient elements as fp32.  `p` is 32-byte aligned for fp32 and 16-byte aligned
+// for bf16.  bf16 -> fp32 is exact: the stored 16 bits become the high half of the fp32 pattern.
+template <bool BF16>
+__device__ __forceinline__ void load8(const void* p, float (&g)[8]) {
+    if constexpr (!BF16) {
+        uint32_t v[8];
+        ldg256_stream(p, v);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) g[i] = __uint_as_float(v[i]);
+    } else {
+        uint4 v;
+        asm volatile("ld.global.nc.L1::no_allocate.v4.b32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            g[2 * i] = __uint_as_float(w[i] << 16);
+            g[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        }
+    }
+}
+
+// One element, any alignment (ragged tails).
+template <bool BF16>
+__device__ __forceinline__ float load1(const void* base, uint64_t j) {
+    if constexpr (!BF16) return __ldg(reinterpret_cast<const float*>(base) + j);
+    else return __uint_as_float(static_cast<uint32_t>(__ldg(reinterpret_cast<const unsigned short*>(base) + j)) << 16);
+}
+
+// ---- Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11) -------------------------------------------
+// Ten rounds; each round multiplies counter words 0 and 2 by fixed odd constants, keeps both halves
+// of the 64-bit products and xors the high halves with the remaining counter words and the round
+// key; the key advances by a Weyl sequence between rounds.
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                              uint32_t k0, uint32_t k1, uint32_t (&out)[4]) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint64_t p0 = static_cast<uint64_t>(0xD2511F53u) * c0;
+        const uint64_t p1 = static_cast<uint64_t>(0xCD9E8D57u) * c2;
+        const uint32_t n0 = static_cast<uint32_t>(p1 >> 32) ^ c1 ^ k0;
+        const uint32_t n2 = static_cast<uint32_t>(p0 >> 32) ^ c3 ^ k1;
+        c1 = static_cast<uint32_t>(p1);
+        c3 = static_cast<uint32_t>(p0);
+        c0 = n0;
+        c2 = n2;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// ---- warp / block reductions -----------------------------------------------------------------------
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+__device__ __forceinline__ unsigned long long warp_sum(unsigned long long v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_down_sync(0xFFFFFFFFu, v, o));
+    return v;
+}
+
+}  // namespace tq

@@ -1,0 +1,167 @@
+"""CPU-side checks of the CUDA library: it loads, exports what include/tq.h declares, its host
+logic (sizes, argument validation, tq_params) behaves, and tq_params agrees with the oracle.
+
+No kernel is launched here; argument errors are detected before any CUDA call is made.
+"""
+import ctypes as C
+import math
+import os
+import re
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def tq():
+    from paper_2402_01798_b200 import build
+    build.build()
+    from paper_2402_01798_b200 import binding
+    binding.lib()
+    return binding
+
+
+def test_library_exports_every_declared_symbol(tq):
+    header = open(os.path.join(ROOT, "include", "tq.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(tq_[a-z_]+)\s*\(", header))
+    assert declared == set(tq.EXPORTS)
+    for name in declared:
+        assert getattr(tq.lib(), name) is not None
+
+
+def test_missing_library_fails_loudly(tq, monkeypatch):
+    monkeypatch.setattr(tq, "_lib", None)
+    monkeypatch.setattr(tq, "LIB_PATH", os.path.join(ROOT, "no_such_dir", "libtq.so"))
+    with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
+        tq.lib()
+
+
+def test_product_does_not_import_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2402_01798_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".cpp", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert not re.search(r"import\s+oracle|from\s+oracle|tq_oracle|orc_[a-z]", text), f
+    text = open(os.path.join(ROOT, "oracle", "tq_oracle.c")).read() + open(os.path.join(ROOT, "oracle", "__init__.py")).read()
+    assert "paper_2402_01798_b200" not in text and "tq.h" not in text
+
+
+def test_struct_sizes_and_packed_words(tq):
+    assert C.sizeof(tq.Stats) == 64 and C.sizeof(tq.Params) == 176
+    for d in (0, 1, 10, 11, 32, 33, 100_000, 100_003, 10**9):
+        for b in (1, 2, 3, 4):
+            assert tq.tq_packed_words(d, b) == (-(-d * b // 32) + 3) // 4 * 4
+    assert tq.tq_packed_words(100_000, 2) == 6252
+    assert tq.tq_packed_words(1_000_000_000, 3) == 93_750_000
+    assert tq.tq_stats_workspace_bytes(1) > 0
+    assert tq.tq_stats_workspace_bytes(16) > tq.tq_stats_workspace_bytes(1)
+
+
+def _stats(cls, **kw):
+    base = dict(d=1_000_000, n_tail=240_000, n_nonfinite=0, sum_abs=1000.0, sum_sq=10.0,
+                sum_log_tail=240_000 / 1.9, max_abs=0.7, g_min=1e-3)
+    base.update(kw)
+    return cls(**base)
+
+
+CASES = [(L, mode, gamma, rule)
+         for L in (2, 4, 8, 16) for mode in (0, 1)
+         for gamma in (2.2, 2.5, 3.0, 3.5, 4.0, 5.0, math.nan)
+         for rule in (0, 1)]
+
+
+@pytest.mark.parametrize("L,mode,gamma,rule", CASES)
+def test_tq_params_agrees_with_oracle(tq, orc, L, mode, gamma, rule):
+    """Library and oracle implement Section 4 separately (both in double, rounded once to fp32);
+    alpha, levels and inverse widths must agree to fp32 rounding, flags exactly."""
+    for kw in (dict(), dict(n_tail=60_000, sum_log_tail=60_000 / 2.6, g_min=3e-3, max_abs=0.05),
+               dict(n_tail=400_000, sum_log_tail=400_000 / 1.3, g_min=2e-4, max_abs=30.0)):
+        a = tq.tq_params(_stats(tq.Stats, **kw), L, mode, gamma, rule)
+        b = orc.params(_stats(orc.Stats, **kw), L, mode, gamma, rule)
+        assert a.bits == b.bits and a.num_levels == b.num_levels == L and a.mode == b.mode == mode
+        assert a.flags == b.flags
+        assert math.isclose(a.alpha, b.alpha, rel_tol=3e-7)
+        assert math.isclose(a.gamma, b.gamma, rel_tol=3e-7) and math.isclose(a.rho, b.rho, rel_tol=3e-7)
+        assert np.allclose(list(a.levels), list(b.levels), rtol=5e-7, atol=0)
+        assert np.allclose(list(a.inv_width), list(b.inv_width), rtol=2e-6, atol=0)
+        assert math.isclose(a.inv_step, b.inv_step, rel_tol=3e-7)
+        lv = np.array(a.levels[:L], dtype=np.float64)
+        assert np.all(np.diff(lv) > 0) and lv[0] == -a.alpha and lv[-1] == a.alpha
+        for k in range(L - 1):                                  # inverse widths are rounded UP
+            assert a.inv_width[k] >= 1.0 / float(np.float32(lv[k + 1] - lv[k]))
+
+
+def test_tq_params_errors(tq):
+    st = _stats(tq.Stats)
+    for bad in (2.0, 1.0, float("inf")):
+        with pytest.raises(tq.TqError) as e:
+            tq.tq_params(st, 8, tq.UNIFORM, bad)
+        assert e.value.status == tq.ERR_DOMAIN
+    with pytest.raises(tq.TqError) as e:
+        tq.tq_params(st, 6, tq.UNIFORM, 3.0)
+    assert e.value.status == tq.ERR_INVALID_ARG
+    with pytest.raises(tq.TqError) as e:
+        tq.tq_params(_stats(tq.Stats, n_tail=0), 8, tq.UNIFORM, 3.0)
+    assert e.value.status == tq.ERR_DOMAIN
+    with pytest.raises(tq.TqError) as e:
+        tq.tq_params(_stats(tq.Stats, g_min=0.0), 8, tq.UNIFORM, 3.0)
+    assert e.value.status == tq.ERR_DOMAIN
+    p = tq.tq_params(st, 8, tq.UNIFORM, 3.0, tq.ALPHA_USER, 0.125)
+    assert p.alpha == 0.125 and p.flags == 0
+    capped = tq.tq_params(_stats(tq.Stats, max_abs=2e-3), 16, tq.NONUNIFORM, 2.2)
+    assert capped.flags & tq.FLAG_ALPHA_CAPPED and capped.alpha == np.float32(2e-3)
+    with pytest.raises(tq.TqError) as e:
+        tq.tq_params_from_levels([-1.0, 0.5, 0.5, 1.0])
+    assert e.value.status == tq.ERR_DEGENERATE_LEVELS
+    with pytest.raises(tq.TqError) as e:
+        tq.tq_params_from_levels([-1.0, 0.0, 0.5, 2.0])
+    assert e.value.status == tq.ERR_DOMAIN
+
+
+def test_params_from_levels_agrees_with_oracle(tq, orc):
+    lv = [-2.0, -0.5, -0.1, -0.01, 0.01, 0.1, 0.5, 2.0]
+    a, b = tq.tq_params_from_levels(lv), orc.table_params(lv)
+    assert list(a.levels) == list(b.levels) and list(a.inv_width) == list(b.inv_width)
+    assert a.alpha == b.alpha == 2.0 and a.inv_step == b.inv_step and a.bits == 3
+
+
+def test_argument_validation_without_a_gpu(tq):
+    """Bad arguments are rejected by status code before any CUDA call."""
+    L = tq.lib()
+    P = tq.tq_params(_stats(tq.Stats), 8, tq.UNIFORM, 3.0)
+    arr = (tq.Params * 2)(P, P)
+    ok_ptr = 0x7000_0000_0000          # never dereferenced: validation comes first
+    # null / range
+    assert L.tq_compress(None, tq.F32, 64, 64, 1, arr, 0, 0, ok_ptr, 8, None) == tq.ERR_INVALID_ARG
+    assert L.tq_compress(ok_ptr, tq.F32, 64, 64, 0, arr, 0, 0, ok_ptr, 8, None) == tq.ERR_INVALID_ARG
+    assert L.tq_compress(ok_ptr, tq.F32, 64, 64, 65, arr, 0, 0, ok_ptr, 8, None) == tq.ERR_INVALID_ARG
+    assert L.tq_compress(ok_ptr, 7, 64, 64, 1, arr, 0, 0, ok_ptr, 8, None) == tq.ERR_INVALID_ARG
+    assert L.tq_compress(ok_ptr, tq.F32, 64, 32, 1, arr, 0, 0, ok_ptr, 8, None) == tq.ERR_INVALID_ARG
+    # alignment
+    assert L.tq_compress(ok_ptr + 4, tq.F32, 64, 64, 1, arr, 0, 0, ok_ptr, 8, None) == tq.ERR_ALIGNMENT
+    assert L.tq_compress(ok_ptr, tq.F32, 60, 60, 2, arr, 0, 0, ok_ptr, 8, None) == tq.ERR_ALIGNMENT
+    assert L.tq_compress(ok_ptr, tq.F32, 64, 64, 1, arr, 0, 0, ok_ptr + 4, 8, None) == tq.ERR_ALIGNMENT
+    assert L.tq_compress(ok_ptr, tq.F32, 64, 64, 1, arr, 0, 0, ok_ptr, 6, None) == tq.ERR_ALIGNMENT
+    # size
+    assert L.tq_compress(ok_ptr, tq.F32, 64, 64, 1, arr, 0, 0, ok_ptr, 4, None) == tq.ERR_BUFFER_TOO_SMALL
+    # mixed bits
+    P4 = tq.tq_params(_stats(tq.Stats), 16, tq.UNIFORM, 3.0)
+    mixed = (tq.Params * 2)(P, P4)
+    assert L.tq_compress(ok_ptr, tq.F32, 64, 64, 2, mixed, 0, 0, ok_ptr, 8, None) == tq.ERR_INVALID_ARG
+    assert L.tq_decompress_aggregate(ok_ptr, 8, 2, 64, mixed, None, ok_ptr, None) == tq.ERR_INVALID_ARG
+    assert L.tq_decompress_aggregate(ok_ptr, 8, 1, 64, arr, None, ok_ptr + 16, None) == tq.ERR_ALIGNMENT
+    assert L.tq_decompress_aggregate(ok_ptr, 4, 1, 64, arr, None, ok_ptr, None) == tq.ERR_BUFFER_TOO_SMALL
+    # stats
+    ws = tq.tq_stats_workspace_bytes(2)
+    assert L.tq_stats(ok_ptr, tq.F32, 64, 64, 2, 0.0, 1.0, ok_ptr, ok_ptr, ws - 1, None) == tq.ERR_BUFFER_TOO_SMALL
+    assert L.tq_stats(ok_ptr, tq.F32, 64, 64, 2, 0.0, 0.0, ok_ptr, ok_ptr, ws, None) == tq.ERR_INVALID_ARG
+    assert L.tq_stats(ok_ptr, tq.F32, 64, 64, 2, 0.0, 1.0, None, ok_ptr, ws, None) == tq.ERR_INVALID_ARG
+    assert L.tq_stats(ok_ptr, tq.F32, 64, 64, 2, 0.0, 1.0, ok_ptr, ok_ptr + 8, ws, None) == tq.ERR_ALIGNMENT
+    # d = 0 needs no device at all
+    assert L.tq_compress(ok_ptr, tq.F32, 0, 0, 1, arr, 0, 0, ok_ptr, 0, None) == tq.OK
+    assert L.tq_decompress_aggregate(ok_ptr, 0, 1, 0, arr, None, ok_ptr, None) == tq.OK
+    assert L.tq_strerror(tq.ERR_ALIGNMENT).decode().startswith("pointer")

@@ -1,0 +1,330 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle.
+
+Chain of custody: every stage is compared on the SAME inputs.  The oracle is handed the very bytes
+the GPU consumed (copied back) and, for the bit-exact stages, the library's own upstream outputs
+(its g_min, its quantizer parameters); each upstream output is itself compared with the oracle's.
+
+Bars: packed words / codes bit-exact; aggregated updates within 1e-6 relative per element (the
+pinned arithmetic actually gives equality, which is asserted too); statistics: counts and max
+exact, sums to the tolerance derived from the kernel's fp32-over-16-elements accumulation.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+F32 = np.float32
+# sums: 16 positive fp32 terms are added before going to fp64: relative error <= 15 * 2^-24 ~ 9e-7,
+# plus 2^-24 for the square.  The logarithm uses the hardware lg2 approximation (absolute error about
+# 2^-22 per term, terms of order one).
+TOL_SUM = 2e-6
+TOL_LOG = 5e-6
+
+
+@pytest.fixture(scope="module")
+def tq():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2402_01798_b200 import binding
+    binding.lib()                    # must be prebuilt and in-tree: no fallback
+    return binding
+
+
+def to_oracle_params(orc, p):
+    q = orc.Params()
+    for f in ("bits", "num_levels", "mode", "flags", "alpha", "inv_step", "gamma", "g_min", "rho", "iterations"):
+        setattr(q, f, getattr(p, f))
+    for k in range(16):
+        q.levels[k] = p.levels[k]
+        q.inv_width[k] = p.inv_width[k]
+    return q
+
+
+def host_f32(orc, t: torch.Tensor) -> np.ndarray:
+    """The bytes the GPU consumed, as the fp32 values the method sees."""
+    if t.dtype == torch.bfloat16:
+        return orc.bf16_to_f32(t.view(torch.int16).cpu().numpy().view(np.uint16))
+    return t.cpu().numpy()
+
+
+def heavy_tailed(d, n, dtype, seed, scale=1e-3, gamma=3.0, device="cuda"):
+    from paper_2402_01798_b200 import inputs
+    stride = inputs.worker_stride(d, dtype)
+    g = torch.zeros((n, stride), dtype=dtype, device=device)
+    for i in range(n):
+        if d:
+            inputs.powerlaw_gradient(d, gamma, scale, seed + i, device, dtype, out=g[i, :d])
+    return g
+
+
+def salt_special_values(g, d, p):
+    """Overwrite a few entries with the degenerate inputs the method has."""
+    vals = [float("nan"), float("inf"), float("-inf"), p.alpha, -p.alpha, 0.0, -0.0,
+            2 * p.alpha, -2 * p.alpha, 1e-38, 3e38] + [p.levels[k] for k in range(p.num_levels)]
+    rng = np.random.default_rng(d)
+    idx = rng.choice(d, size=min(d, len(vals)), replace=False)
+    for i, v in zip(idx, vals):
+        g[:, int(i)] = v
+
+
+def lib_params_for(tq, g, d, L, mode, gamma, rule=None):
+    st = tq.stats_to_host(tq.tq_stats(g, d))
+    rule = tq.ALPHA_FIXED_POINT if rule is None else rule
+    return st, [tq.tq_params(s, L, mode, gamma, rule) for s in st]
+
+
+# ----------------------------------------------------------------------------------------- stats
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("d,n", [(0, 1), (1, 1), (15, 2), (16, 1), (17, 3), (4099, 2), (100_003, 3), (3_000_000, 4)])
+def test_stats_parity(tq, orc, d, n, dtype):
+    g = heavy_tailed(d, n, dtype, seed=d + 1)
+    if d > 40:
+        g[:, 7] = float("nan"); g[:, 33] = float("inf"); g[0, 21] = float("-inf")
+    for g_min_in in (0.0, 7e-4):
+        for kappa in ((1.0, 2.5) if g_min_in == 0.0 else (1.0,)):
+            got = tq.stats_to_host(tq.tq_stats(g, d, g_min=g_min_in, kappa=kappa))
+            assert len(got) == n
+            for i in range(n):
+                x = host_f32(orc, g[i, :d])
+                auto = orc.stats(x, g_min=g_min_in, kappa=kappa)          # oracle's own threshold
+                s = got[i]
+                assert s.d == d and s.n_nonfinite == auto.n_nonfinite and s.max_abs == auto.max_abs
+                assert math.isclose(s.sum_abs, auto.sum_abs, rel_tol=TOL_SUM, abs_tol=0)
+                assert math.isclose(s.sum_sq, auto.sum_sq, rel_tol=TOL_SUM, abs_tol=0)
+                assert math.isclose(s.g_min, auto.g_min, rel_tol=TOL_SUM, abs_tol=0)
+                if g_min_in > 0:
+                    assert s.g_min == F32(g_min_in)
+                ref = orc.stats(x, g_min=s.g_min) if s.g_min > 0 else auto   # tail part on the library's g_min
+                assert s.n_tail == ref.n_tail
+                assert math.isclose(s.sum_log_tail, ref.sum_log_tail, rel_tol=TOL_LOG, abs_tol=1e-9)
+
+
+def test_stats_is_deterministic_and_reuses_workspace(tq):
+    g = heavy_tailed(1_000_003, 4, torch.float32, seed=3)
+    ws = torch.empty(tq.tq_stats_workspace_bytes(4), dtype=torch.uint8, device="cuda")
+    ws.fill_(0xAB)                                        # scratch contents need not be initialised
+    a = tq.tq_stats(g, 1_000_003, workspace=ws).cpu()
+    b = tq.tq_stats(g, 1_000_003, workspace=ws).cpu()
+    c = tq.tq_stats(g, 1_000_003).cpu()
+    assert torch.equal(a, b) and torch.equal(a, c)
+
+
+# -------------------------------------------------------------------------------------- compress
+SIZES = [1, 3, 8, 31, 32, 33, 127, 255, 256, 257, 8191, 8192, 8193, 100_003]
+
+
+@pytest.mark.parametrize("bits", [1, 2, 3, 4])
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_compress_bit_exact_ragged_sizes(tq, orc, bits, mode, dtype):
+    L = 1 << bits
+    for d in SIZES:
+        n = 1 if d % 2 else 3
+        g = heavy_tailed(d, n, dtype, seed=100 * bits + d)
+        st = [orc.stats(host_f32(orc, g[i, :d]), g_min=5e-4) for i in range(n)]
+        ps = []
+        for i, s in enumerate(st):                        # parameters from the library's host code
+            ls = tq.Stats(d=max(s.d, 1000), n_tail=max(s.n_tail, 100), n_nonfinite=0, sum_abs=s.sum_abs, sum_sq=s.sum_sq,
+                          sum_log_tail=max(s.sum_log_tail, 50.0), max_abs=max(s.max_abs, 0.05), g_min=5e-4)
+            ps.append(tq.tq_params(ls, L, mode, 3.0 + 0.25 * i))
+        if d >= 64:
+            salt_special_values(g, d, ps[0])
+        seed, first = 0xC0FFEE123456789, 5
+        words = tq.tq_packed_words(d, bits)
+        packed = torch.full((n, words + 8), 0x5A5A5A5A, dtype=torch.int32, device="cuda")   # canary beyond the row
+        tq.tq_compress(g, ps, seed, first, d=d, packed=packed)
+        got = packed.cpu().numpy().view(np.uint32)
+        for i in range(n):
+            want = orc.compress(host_f32(orc, g[i, :d]), to_oracle_params(orc, ps[i]), seed, first + i)
+            assert want.size == words
+            assert np.array_equal(got[i, :words], want), (d, i)
+            assert np.all(got[i, words:] == 0x5A5A5A5A)    # nothing written past the row's words
+
+
+@pytest.mark.parametrize("bits,mode", [(2, 0), (3, 1), (4, 1), (4, 0)])
+def test_compress_million_elements_and_seed_sensitivity(tq, orc, bits, mode):
+    d, n = 1_000_000 + 37, 2
+    g = heavy_tailed(d, n, torch.float32, seed=bits)
+    _, ps = lib_params_for(tq, g, d, 1 << bits, mode, 3.0)
+    a = tq.tq_compress(g, ps, seed=11, d=d).cpu().numpy().view(np.uint32)
+    for i in range(n):
+        assert np.array_equal(a[i], orc.compress(host_f32(orc, g[i, :d]), to_oracle_params(orc, ps[i]), 11, i))
+    b = tq.tq_compress(g, ps, seed=12, d=d).cpu().numpy().view(np.uint32)
+    c = tq.tq_compress(g, ps, seed=11, d=d).cpu().numpy().view(np.uint32)
+    assert not np.array_equal(a, b) and np.array_equal(a, c)
+    # worker index enters the counter: row 1 compressed as "first_worker = 1" equals row 1 of the batch
+    single = tq.tq_compress(g[1:2], ps[1:2], seed=11, first_worker=1, d=d).cpu().numpy().view(np.uint32)
+    assert np.array_equal(single[0], a[1])
+
+
+def test_uniform_table_through_nonuniform_kernel(tq, orc):
+    """A uniform codebook pushed through the table-search path yields a valid code stream for the same
+    quantizer: identical intervals except within rounding of a level (where both answers are the
+    paper's quantizer), so the dequantized values differ by less than one ulp-scale amount."""
+    d = 200_000
+    g = heavy_tailed(d, 1, torch.float32, seed=9)
+    _, (pu,) = lib_params_for(tq, g, d, 8, tq.UNIFORM, 3.0)
+    pt = tq.tq_params_from_levels([pu.levels[k] for k in range(8)], tq.NONUNIFORM)
+    cu = orc.unpack(tq.tq_compress(g, [pu], 3, d=d).cpu().numpy().view(np.uint32)[0], d, 3)
+    ct = orc.unpack(tq.tq_compress(g, [pt], 3, d=d).cpu().numpy().view(np.uint32)[0], d, 3)
+    assert np.mean(cu != ct) < 1e-4
+    want = orc.compress(host_f32(orc, g[0, :d]), to_oracle_params(orc, pt), 3, 0)
+    assert np.array_equal(orc.unpack(want, d, 3), ct)
+
+
+# ---------------------------------------------------------------------------- decompress-aggregate
+@pytest.mark.parametrize("bits", [1, 2, 3, 4])
+@pytest.mark.parametrize("n", [1, 2, 3, 5, 8, 16, 33])
+def test_decompress_aggregate_exact(tq, orc, bits, n):
+    L = 1 << bits
+    rng = np.random.default_rng(bits * 100 + n)
+    for d in (1, 7, 8, 31, 32, 33, 255, 257, 4099, 100_003):
+        words = tq.tq_packed_words(d, bits)
+        codes = rng.integers(0, L, (n, d), dtype=np.uint8)
+        packed_h = np.stack([orc.pack(codes[i], bits) for i in range(n)])
+        ps = []
+        for i in range(n):
+            a = 0.01 * (1 + 0.3 * i)
+            mags = np.geomspace(a / 50, a, L // 2).astype(F32) if L > 2 else np.array([a], dtype=F32)
+            lv = np.concatenate([-mags[::-1], mags])
+            ps.append(tq.tq_params_from_levels([float(x) for x in lv]))
+        packed = torch.from_numpy(packed_h.view(np.int32)).cuda()
+        out = torch.full((d + 16,), 777.0, dtype=torch.float32, device="cuda")
+        tq.tq_decompress_aggregate(packed, d, ps, out=out)
+        got = out.cpu().numpy()
+        want = orc.decompress_aggregate(packed_h, d, [to_oracle_params(orc, p) for p in ps])
+        assert np.all(np.abs(got[:d] - want) <= 1e-6 * np.maximum(np.abs(got[:d]), np.abs(want)))
+        assert np.array_equal(got[:d], want)
+        assert np.all(got[d:] == 777.0)                    # no write past d
+        if n in (3, 8) and d in (33, 4099):
+            w = rng.random(n).astype(F32); w /= w.sum()
+            gw = tq.tq_decompress_aggregate(packed, d, ps, weights=list(w)).cpu().numpy()
+            ww = orc.decompress_aggregate(packed_h, d, [to_oracle_params(orc, p) for p in ps], weights=w)
+            assert np.array_equal(gw, ww)
+
+
+# ------------------------------------------------------------------------------- whole round trips
+def run_round(tq, g, d, L, mode, gamma, seed):
+    st, ps = lib_params_for(tq, g, d, L, mode, gamma)
+    packed = tq.tq_compress(g, ps, seed, d=d)
+    out = tq.tq_decompress_aggregate(packed, d, ps)
+    torch.cuda.synchronize()
+    return st, ps, packed, out
+
+
+def check_params_against_oracle(tq, orc, st, ps, L, mode, gamma):
+    for s, p in zip(st, ps):
+        o = orc.params(orc.Stats(d=s.d, n_tail=s.n_tail, n_nonfinite=s.n_nonfinite, sum_abs=s.sum_abs, sum_sq=s.sum_sq,
+                                 sum_log_tail=s.sum_log_tail, max_abs=s.max_abs, g_min=s.g_min), L, mode, gamma)
+        assert o.flags == p.flags and math.isclose(o.alpha, p.alpha, rel_tol=3e-7)
+        assert np.allclose(list(o.levels), list(p.levels), rtol=5e-7, atol=0)
+
+
+def test_config1_small_full(tq, orc):
+    """d = 100,000, N = 1, gamma = 3, scale 1e-3, uniform, 4 levels: everything compared in full."""
+    from paper_2402_01798_b200 import inputs
+    w = inputs.WORKLOADS[0]
+    g, _ = inputs.make_worker_gradients(w, "cuda")
+    st, ps, packed, out = run_round(tq, g, w.d, w.num_levels, tq.UNIFORM, w.gamma, seed=0)
+    x = host_f32(orc, g[0, :w.d])
+    o = orc.stats(x)
+    assert st[0].n_nonfinite == 0 and st[0].max_abs == o.max_abs
+    assert math.isclose(st[0].sum_abs, o.sum_abs, rel_tol=TOL_SUM) and math.isclose(st[0].g_min, o.g_min, rel_tol=TOL_SUM)
+    check_params_against_oracle(tq, orc, st, ps, 4, orc.UNIFORM, w.gamma)
+    op = to_oracle_params(orc, ps[0])
+    want = orc.compress(x, op, 0, 0)
+    assert packed.shape == (1, 6252) and np.array_equal(packed.cpu().numpy().view(np.uint32)[0], want)
+    agg = orc.decompress_aggregate(want[None, :], w.d, [op])
+    assert np.array_equal(out.cpu().numpy(), agg)
+
+
+@pytest.mark.parametrize("cfg", [1, 2])
+def test_config2_config3_full_size(tq, orc, cfg):
+    """d = 11.2 M x 8 workers (uniform, 8 levels) and d = 25.6 M x 16 workers (non-uniform, 16 levels) at
+    full size, in the launch configuration the benchmark times.  Packed rows are compared in full for
+    two workers and on windows for the rest; the aggregate is compared on windows (each output needs
+    all N rows)."""
+    from paper_2402_01798_b200 import inputs
+    w = inputs.WORKLOADS[cfg]
+    mode = tq.NONUNIFORM if w.mode == "nonuniform" else tq.UNIFORM
+    g, _ = inputs.make_worker_gradients(w, "cuda")
+    st, ps, packed, out = run_round(tq, g, w.d, w.num_levels, mode, w.gamma, seed=cfg)
+    check_params_against_oracle(tq, orc, st, ps, w.num_levels, mode, w.gamma)
+    ops = [to_oracle_params(orc, p) for p in ps]
+    bits = ps[0].bits
+    for i in (0, w.n_workers - 1):
+        want = orc.compress(host_f32(orc, g[i, :w.d]), ops[i], cfg, i)
+        assert np.array_equal(packed[i].cpu().numpy().view(np.uint32), want), i
+    check_windows(tq, orc, g, w.d, ops, packed, out, seed=cfg, bits=bits, n_windows=6, win=1 << 16)
+
+
+def check_windows(tq, orc, g, d, ops, packed, out, seed, bits, n_windows, win, first_worker=0):
+    """Compare codes and aggregates on 32-aligned windows (start, end, and seeded interior offsets,
+    including one that straddles the 2^32-bit offset of the stream when the row is long enough)."""
+    n = len(ops)
+    rng = np.random.default_rng(seed + 12345)
+    starts = [0, max(0, (d - win) // 32 * 32)]
+    if d * bits > 2 ** 32 + win * bits:
+        starts.append(((2 ** 32 // bits) - win // 2) // 32 * 32)
+    if d > 2 ** 31 + win:
+        starts.append((2 ** 31 - win // 2) // 32 * 32)
+    while len(starts) < n_windows:
+        starts.append(int(rng.integers(0, max(1, d - win))) // 32 * 32)
+    for a in starts:
+        b = min(d, a + win)
+        w0, w1 = a * bits // 32, -(-b * bits // 32)
+        rows = packed[:, w0:w1].cpu().numpy().view(np.uint32)
+        for i in range(n):
+            x = host_f32(orc, g[i, a:b])
+            want = orc.pack(orc.quantize_window(x, a, ops[i], seed, first_worker + i), bits, words=w1 - w0)
+            assert np.array_equal(rows[i], want), (a, i)
+        agg = orc.decompress_aggregate(np.ascontiguousarray(rows), b - a, ops)
+        got = out[a:b].cpu().numpy()
+        assert np.all(np.abs(got - agg) <= 1e-6 * np.maximum(np.abs(got), np.abs(agg)))
+        assert np.array_equal(got, agg), a
+
+
+@pytest.mark.parametrize("gamma,mode,L", [(2.2, "uniform", 4), (3.0, "nonuniform", 16), (4.0, "nonuniform", 4), (2.2, "nonuniform", 16)])
+def test_config4_bf16_outliers_windows(tq, orc, gamma, mode, L):
+    """d = 124 M bf16 x 8 workers with 1% of entries multiplied by 100: full-size launch, windows compared.
+    (gamma = 2.2 with 16 non-uniform levels has no finite fixed point: alpha is capped at max|g|.)"""
+    from paper_2402_01798_b200 import inputs
+    w = next(c for c in inputs.CONFIG4_SWEEP if c.gamma == gamma and c.mode == mode and c.num_levels == L)
+    m = tq.NONUNIFORM if mode == "nonuniform" else tq.UNIFORM
+    g, _ = inputs.make_worker_gradients(w, "cuda")
+    st, ps, packed, out = run_round(tq, g, w.d, L, m, gamma, seed=44)
+    check_params_against_oracle(tq, orc, st, ps, L, m, gamma)
+    if gamma == 2.2 and mode == "nonuniform" and L == 16:
+        assert all(p.flags & tq.FLAG_ALPHA_CAPPED for p in ps)
+    # statistics of one full row against the oracle
+    x = host_f32(orc, g[3, :w.d])
+    o = orc.stats(x, g_min=st[3].g_min)
+    assert st[3].n_tail == o.n_tail and st[3].max_abs == o.max_abs
+    assert math.isclose(st[3].sum_abs, o.sum_abs, rel_tol=TOL_SUM) and math.isclose(st[3].sum_log_tail, o.sum_log_tail, rel_tol=TOL_LOG)
+    del x
+    check_windows(tq, orc, g, w.d, [to_oracle_params(orc, p) for p in ps], packed, out, seed=44, bits=ps[0].bits,
+                  n_windows=5, win=1 << 16)
+
+
+def test_config5_billion_elements_windows(tq, orc):
+    """d = 10^9 x 4 workers, non-uniform, 8 levels (3-bit codes crossing word boundaries; element and
+    bit offsets beyond 2^32): full-size launch; windows at both ends, across the 2^32-bit offset, and
+    at seeded interior offsets."""
+    from paper_2402_01798_b200 import inputs
+    w = inputs.WORKLOADS[4]
+    g, _ = inputs.make_worker_gradients(w, "cuda")
+    st, ps, packed, out = run_round(tq, g, w.d, w.num_levels, tq.NONUNIFORM, w.gamma, seed=5)
+    check_params_against_oracle(tq, orc, st, ps, 8, tq.NONUNIFORM, w.gamma)
+    assert all(s.d == w.d and s.n_nonfinite == 0 for s in st)
+    assert packed.shape == (4, 93_750_000)
+    check_windows(tq, orc, g, w.d, [to_oracle_params(orc, p) for p in ps], packed, out, seed=5, bits=3,
+                  n_windows=7, win=1 << 16)
+    # statistics of one full row (10^9 elements) against the oracle
+    x = host_f32(orc, g[1, :w.d])
+    o = orc.stats(x, g_min=st[1].g_min)
+    assert st[1].n_tail == o.n_tail and st[1].max_abs == o.max_abs
+    assert math.isclose(st[1].sum_abs, o.sum_abs, rel_tol=TOL_SUM) and math.isclose(st[1].sum_sq, o.sum_sq, rel_tol=TOL_SUM)
+    assert math.isclose(st[1].sum_log_tail, o.sum_log_tail, rel_tol=TOL_LOG)
