@@ -20,7 +20,6 @@ import argparse
 import json
 import os
 import statistics
-import subprocess
 import sys
 import threading
 import time
@@ -43,60 +42,55 @@ def hbm_peak():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
-    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Samples SM clocks and throttle reasons through NVML (read-only) while the timed region runs."""
 
-    def __init__(self, index: int):
-        self.index, self.proc, self.lines = index, None, []
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.index, self.period, self.samples, self.reasons = index, period_s, [], set()
+        self.max_mhz, self.stop_flag, self.thread, self.err = None, False, None, None
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
-                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.thread = threading.Thread(target=self._pump, daemon=True)
-            self.thread.start()
-        except Exception:
-            self.proc = None
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            idx = self.index
+            if visible:
+                ids = [v.strip() for v in visible.split(",") if v.strip()]
+                if idx < len(ids) and ids[idx].isdigit():
+                    idx = int(ids[idx])
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(idx)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception as e:            # no NVML: report that instead of clocks
+            self.err = repr(e)
+            return
+        self.thread = threading.Thread(target=self._run, daemon=True)
+        self.thread.start()
 
-    def _pump(self):
-        for line in self.proc.stdout:
-            self.lines.append(line.strip())
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
+        while not self.stop_flag:
+            try:
+                self.samples.append(float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for nm, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(nm)
+            except Exception as e:
+                self.err = repr(e)
+                break
+            time.sleep(self.period)
 
     def stop(self):
-        if not self.proc:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        sm, mx, reasons = [], [], set()
-        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
-        for line in self.lines:
-            parts = [p.strip() for p in line.split(",")]
-            if len(parts) < 6:
-                continue
-            try:
-                sm.append(float(parts[0])); mx.append(float(parts[1]))
-            except ValueError:
-                continue
-            for nm, val in zip(names, parts[2:6]):
-                if val.lower().startswith("active"):
-                    reasons.add(nm)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
-
-
-def oracle_params_from(oracle, p):
-    q = oracle.Params()
-    for f in ("bits", "num_levels", "mode", "flags", "alpha", "inv_step", "gamma", "g_min", "rho", "iterations"):
-        setattr(q, f, getattr(p, f))
-    for k in range(16):
-        q.levels[k] = p.levels[k]
-        q.inv_width[k] = p.inv_width[k]
-    return q
+        self.stop_flag = True
+        if self.thread:
+            self.thread.join(timeout=2)
+        out = {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz,
+               "samples": len(self.samples), "reasons": sorted(self.reasons)}
+        if self.err:
+            out["error"] = self.err
+        return out
 
 
 def cpu_oracle_round(w, sample_d: int, seed: int = 0):
@@ -135,9 +129,10 @@ def run_reference(args, w):
     if rank != 0:
         return
     esz = 2 if w.dtype == torch.bfloat16 else 4
-    sample_d = min(w.d, max(1 << 16, (1 << 25) // w.n_workers))      # about 33 M elements per step
+    # bounded sample: about 1.5e9 element-rounds over the whole run (a couple of minutes of one core)
+    sample_d = min(w.d, max(1 << 16, int(1.5e9 / max(args.steps + args.warmup, 1)) // w.n_workers))
     for _ in range(args.warmup):
-        cpu_oracle_round(w, min(sample_d, 1 << 16))
+        cpu_oracle_round(w, sample_d)
     times = [cpu_oracle_round(w, sample_d) for _ in range(args.steps)]
     t = sum(times) / len(times)
     val = w.n_workers * sample_d * esz / t / 1e9
@@ -158,7 +153,7 @@ def run_reference(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=2, help="index into the five workloads (default: 25.6M x 16)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
