@@ -36,6 +36,7 @@ extern "C" {
 
 #define TQ_MAX_LEVELS 16
 #define TQ_MAX_WORKERS 64
+#define TQ_STATIC_MAX_WORKERS 16   /* most workers one tq_stats_static call can reduce */
 
 typedef enum {
     TQ_OK = 0,
@@ -44,7 +45,8 @@ typedef enum {
     TQ_ERR_ALIGNMENT = -3,         /* a device pointer or stride misses its stated alignment */
     TQ_ERR_BUFFER_TOO_SMALL = -4,  /* packed stride or workspace smaller than required */
     TQ_ERR_DEGENERATE_LEVELS = -5, /* codebook not strictly increasing in fp32 */
-    TQ_ERR_CUDA = -6               /* a CUDA runtime call failed; see tq_last_cuda_error */
+    TQ_ERR_CUDA = -6,              /* a CUDA runtime call failed; see tq_last_cuda_error */
+    TQ_ERR_STATIC_LIMIT = -7       /* request exceeds the library's built-in scratch (tq_stats_static) */
 } tq_status;
 
 typedef enum { TQ_F32 = 0, TQ_BF16 = 1 } tq_dtype;               /* gradient storage type */
@@ -113,6 +115,30 @@ size_t tq_stats_workspace_bytes(uint32_t n_workers);
 tq_status tq_stats(const void* grad_dev, tq_dtype dtype, uint64_t d, uint64_t grad_stride,
                    uint32_t n_workers, float g_min, float kappa, tq_stats_t* stats_dev,
                    void* workspace_dev, size_t ws_bytes, void* stream);
+
+/*
+ * tq_stats without a scratch argument, for callers that cannot allocate device memory.
+ * (The paper has no counterpart; this is a packaging variant of tq_stats, same kernels, same results.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a framework's stream-ordered
+ * or pooled allocator callback, in a plugin that is handed device buffers but owns none, or in a
+ * latency-critical loop where an allocation would synchronise the device.  Such a caller still passes
+ * its gradient and the output records; only the reduction's scratch (block partials + tickets) comes
+ * from the library: a fixed 1 MiB + 384 B array that lives in the library's device image, so every GPU
+ * that loads libtq holds it until the process exits.
+ *
+ *   n_workers    at most TQ_STATIC_MAX_WORKERS (16); more returns TQ_ERR_STATIC_LIMIT and does nothing.
+ *   all other arguments, results and errors as for tq_stats.
+ *
+ * The call allocates nothing and frees nothing.  The first call on each device looks up the array's
+ * device address (once per device, with that device current); make that first call outside any
+ * stream capture.  All calls on a device share the one array and it keeps the previous call's
+ * contents: the library clears the ticket counters itself at the start of every call, nothing else
+ * needs to start at zero.  Two calls whose kernels overlap on the same GPU (different streams, or
+ * different host threads) race on the array and give wrong statistics: serialise them.
+ */
+tq_status tq_stats_static(const void* grad_dev, tq_dtype dtype, uint64_t d, uint64_t grad_stride,
+                          uint32_t n_workers, float g_min, float kappa, tq_stats_t* stats_dev, void* stream);
 
 /*
  * Parameter design on the host (Section 4), O(L) work in double precision.

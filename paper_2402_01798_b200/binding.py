@@ -18,12 +18,14 @@ LIB_PATH = os.path.join(_PKG, "libtq.so")
 MAX_LEVELS, MAX_WORKERS = 16, 64
 OK, ERR_INVALID_ARG, ERR_DOMAIN, ERR_ALIGNMENT, ERR_BUFFER_TOO_SMALL, ERR_DEGENERATE_LEVELS, ERR_CUDA = \
     0, -1, -2, -3, -4, -5, -6
+ERR_STATIC_LIMIT = -7
+STATIC_MAX_WORKERS = 16
 F32, BF16 = 0, 1
 UNIFORM, NONUNIFORM = 0, 1
 ALPHA_CLOSED, ALPHA_FIXED_POINT, ALPHA_USER = 0, 1, 2
 FLAG_ALPHA_CAPPED, FLAG_ALPHA_AT_GMIN, FLAG_GAMMA_FROM_MLE = 1, 2, 4
 
-EXPORTS = ("tq_packed_words", "tq_stats_workspace_bytes", "tq_stats", "tq_params", "tq_params_from_levels",
+EXPORTS = ("tq_packed_words", "tq_stats_workspace_bytes", "tq_stats", "tq_stats_static", "tq_params", "tq_params_from_levels",
            "tq_compress", "tq_decompress_aggregate", "tq_strerror", "tq_last_cuda_error", "tq_kernel_launches")
 
 
@@ -67,6 +69,7 @@ def lib() -> C.CDLL:
         L.tq_packed_words.argtypes = [u64, u32]; L.tq_packed_words.restype = sz
         L.tq_stats_workspace_bytes.argtypes = [u32]; L.tq_stats_workspace_bytes.restype = sz
         L.tq_stats.argtypes = [vp, C.c_int, u64, u64, u32, f32, f32, vp, vp, sz, vp]; L.tq_stats.restype = C.c_int
+        L.tq_stats_static.argtypes = [vp, C.c_int, u64, u64, u32, f32, f32, vp, vp]; L.tq_stats_static.restype = C.c_int
         L.tq_params.argtypes = [C.POINTER(Stats), u32, C.c_int, f64, C.c_int, f64, C.POINTER(Params)]
         L.tq_params.restype = C.c_int
         L.tq_params_from_levels.argtypes = [C.POINTER(f32), u32, C.c_int, C.POINTER(Params)]
@@ -140,6 +143,19 @@ def tq_stats(grad: torch.Tensor, d: Optional[int] = None, g_min: float = 0.0, ka
         workspace = torch.empty(tq_stats_workspace_bytes(n), dtype=torch.uint8, device=grad.device)
     _check(lib().tq_stats(grad.data_ptr(), _dtype_code(grad), d, stride, n, g_min, kappa, stats_dev.data_ptr(),
                           workspace.data_ptr(), workspace.numel(), _stream(stream)), "tq_stats")
+    return stats_dev
+
+
+def tq_stats_static(grad: torch.Tensor, stats_dev: torch.Tensor, d: Optional[int] = None, g_min: float = 0.0,
+                    kappa: float = 1.0, stream=None) -> torch.Tensor:
+    """tq_stats for callers that cannot allocate: the scratch is the library's own fixed array.
+
+    The caller passes the gradient and the output records (``stats_dev``, n_workers * 64 bytes); this
+    wrapper allocates nothing either.  At most STATIC_MAX_WORKERS rows; calls that overlap on the GPU race.
+    """
+    n, d, stride = _grad_layout(grad, d)
+    _check(lib().tq_stats_static(grad.data_ptr(), _dtype_code(grad), d, stride, n, g_min, kappa,
+                                 stats_dev.data_ptr(), _stream(stream)), "tq_stats_static")
     return stats_dev
 
 

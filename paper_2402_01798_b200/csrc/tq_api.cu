@@ -69,6 +69,23 @@ tq_status tq_stats(const void* grad_dev, tq_dtype dtype, uint64_t d, uint64_t gr
     return e == cudaSuccess ? TQ_OK : cuda_failed(e);
 }
 
+tq_status tq_stats_static(const void* grad_dev, tq_dtype dtype, uint64_t d, uint64_t grad_stride, uint32_t n_workers,
+                          float g_min, float kappa, tq_stats_t* stats_dev, void* stream) {
+    if (tq_status s = check_grad(grad_dev, dtype, d, grad_stride, n_workers)) return s;
+    if (n_workers > TQ_STATIC_MAX_WORKERS) return TQ_ERR_STATIC_LIMIT;
+    if (!stats_dev) return TQ_ERR_INVALID_ARG;
+    if (!(g_min > 0.0f) && !(kappa > 0.0f)) return TQ_ERR_INVALID_ARG;
+    if (!aligned(stats_dev, 8)) return TQ_ERR_ALIGNMENT;
+    tq::StatsCall c{grad_dev, dtype == TQ_BF16, d, grad_stride, n_workers, g_min, kappa, stats_dev, nullptr,
+                    static_cast<cudaStream_t>(stream)};
+    int launched = 0;
+    bool limit = false;
+    const cudaError_t e = tq::launch_stats_static(c, &launched, &limit);
+    if (limit) return TQ_ERR_STATIC_LIMIT;
+    g_launches += static_cast<uint64_t>(launched);
+    return e == cudaSuccess ? TQ_OK : cuda_failed(e);
+}
+
 tq_status tq_compress(const void* grad_dev, tq_dtype dtype, uint64_t d, uint64_t grad_stride, uint32_t n_workers,
                       const tq_params_t* params_host, uint64_t seed, uint32_t first_worker, uint32_t* packed_dev,
                       size_t words_stride, void* stream) {
@@ -119,6 +136,7 @@ const char* tq_strerror(tq_status s) {
         case TQ_ERR_BUFFER_TOO_SMALL: return "buffer too small";
         case TQ_ERR_DEGENERATE_LEVELS: return "codebook not strictly increasing in fp32";
         case TQ_ERR_CUDA: return "CUDA runtime error";
+        case TQ_ERR_STATIC_LIMIT: return "more workers than the built-in scratch of tq_stats_static holds (16)";
     }
     return "unknown status";
 }

@@ -30,5 +30,8 @@ struct StatsCall {
 // Enqueues the reduction; *launches receives the number of kernels launched.
 cudaError_t launch_stats(const StatsCall& c, int* launches);
 size_t stats_workspace_bytes(uint32_t n_workers);
+// Same reduction with the library's built-in scratch array as workspace (c.workspace is ignored).
+// *limit is set when n_workers exceeds what the array holds; nothing is launched then.
+cudaError_t launch_stats_static(const StatsCall& c, int* launches, bool* limit);
 
 }  // namespace tq

@@ -15,6 +15,8 @@
 // HBM traffic per element and pass: 4 bytes (fp32) or 2 bytes (bf16) read.
 #include <math_constants.h>
 
+#include <mutex>
+
 #include "tq_device.cuh"
 #include "tq_launch.h"
 
@@ -210,6 +212,43 @@ cudaError_t launch_stats(const StatsCall& c, int* launches) {
     e = c.bf16 ? launch<true, kTail>(c, grid, partials, tickets) : launch<false, kTail>(c, grid, partials, tickets);
     *launches = 2;
     return e;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Built-in scratch for callers that cannot allocate: enough for TQ_STATIC_MAX_WORKERS workers.
+// It is part of the library's device image (one copy per GPU that loads the library).
+constexpr size_t kStaticScratchBytes =
+    static_cast<size_t>(TQ_STATIC_MAX_WORKERS) * kMaxBlocksPerWorker * sizeof(Partial) + TQ_STATIC_MAX_WORKERS * 2 * sizeof(uint32_t) + 256;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+cudaError_t launch_stats_static(const StatsCall& c, int* launches, bool* limit) {
+    *launches = 0;
+    *limit = c.n_workers > TQ_STATIC_MAX_WORKERS || stats_workspace_bytes(c.n_workers) > kStaticScratchBytes;
+    if (*limit) return cudaSuccess;
+
+    // In host code `g_static_scratch` is only a handle for the symbol, not a device address: the
+    // address must be asked for, per device, with that device current.  Done on the first call
+    // on each device and remembered.
+    constexpr int kMaxDevices = 64;
+    static void* s_addr[kMaxDevices] = {};
+    static std::mutex s_lock;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    void* ptr = nullptr;
+    {
+        std::lock_guard<std::mutex> hold(s_lock);
+        if (!s_addr[dev]) {
+            e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+            if (e != cudaSuccess) return e;
+            s_addr[dev] = ptr;
+        }
+        ptr = s_addr[dev];
+    }
+    StatsCall with_scratch = c;
+    with_scratch.workspace = ptr;
+    return launch_stats(with_scratch, launches);   // clears the tickets first, as every call does
 }
 
 }  // namespace tq
