@@ -1,19 +1,38 @@
 // Client side of Algorithm 1: truncate (Section 3.1, truncation equation), stochastically round onto
 // the codebook (Section 3.1, quantizer equation) and pack b-bit codes, fused in one pass.
 //
-// Work split: a thread owns a run of 32 consecutive elements of one worker = four groups of 8.
-// A group is the unit of randomness: one Philox4x32-10 call (counter = group index, worker) yields
-// 128 bits = eight 16-bit slots, one per element.  A run packs into exactly `bits` 32-bit words, so
-// no thread ever shares a word with another and no shuffles or atomics are needed.
+// Work split: persistent blocks walk tiles of 8192 elements of one worker; in a tile a thread owns a
+// run of 32 consecutive elements = four groups of 8.  A group is the unit of randomness: one
+// Philox4x32-10 call (counter = group index, worker) yields 128 bits = eight 16-bit slots, one per
+// element.  A run packs into exactly `bits` 32-bit words, so no thread ever shares a word with
+// another and no shuffles or atomics are needed.
 // HBM traffic per element: 4 (fp32) or 2 (bf16) bytes read, bits/8 bytes written.
+//
+// The kernel is bound by instruction issue, and within that by the half-rate integer/compare pipe,
+// so the per-element arithmetic is arranged to run on the fp32 multiply-add pipe wherever the
+// result is provably the same:
+//   - floor / int conversion: add 2^23 rounding down, the integer appears in the mantissa;
+//   - threshold T = rint(p * 2^16): one fused multiply-add with 2^23;
+//   - the random slot r as the float 2^23 + r: one byte-permute; [r < T] = sat((2^23 + T) - (2^23 + r)),
+//     a saturating subtract of two exactly representable integers;
+//   - codes are kept as small floats and packed by exact multiply-adds (sums stay below 2^24);
+//   - table offsets are formed as denormal floats whose bit pattern IS the byte offset.
+#include <cmath>
+
 #include "tq_device.cuh"
 #include "tq_launch.h"
 
 namespace tq {
 
+constexpr int kMaxGridCells = 2048;   // finest lookup grid for the non-uniform interval search
+constexpr int kMinGridCells = 32;
+
 // Per-worker quantizer as the kernel sees it.
 struct WorkerQ {
     float alpha, inv_step, top;   // top = (float)(L-1)
+    float inv_2alpha;             // maps [-alpha, alpha] to [0, 1] for the lookup grid
+    float cell_scale;             // grid cells M as the denormal M * 2^-149
+    uint32_t cells;               // M
     float levels[TQ_MAX_LEVELS];
     float inv_width[TQ_MAX_LEVELS];
 };
@@ -21,11 +40,30 @@ struct CompressArgs {
     WorkerQ q[TQ_MAX_WORKERS];
 };
 
-// Round-up decision.  T = rint(p * 2^16) is read from the mantissa of p * 2^16 + 2^23 (one fused
-// rounding, ties to even); the element rounds up iff its 16 random bits r satisfy r < T.
-__device__ __forceinline__ uint32_t rounds_up(float p, uint32_t r16) {
-    const float pm = __fmaf_rn(p, 65536.0f, kMagic);
-    return __float_as_uint(pm) > (r16 + kMagicBits) ? 1u : 0u;
+enum Search { kUniform = 0, kGrid = 1, kBinary = 2 };
+
+__device__ __forceinline__ float mul_sat(float a, float b) {
+    float r; asm("mul.rn.sat.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b)); return r;
+}
+__device__ __forceinline__ float sub_sat(float a, float b) {
+    float r; asm("sub.rn.sat.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b)); return r;
+}
+__device__ __forceinline__ float set_ge(float a, float b) {   // 1.0f if a >= b else 0.0f (0 for NaN)
+    float r; asm("set.ge.f32.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b)); return r;
+}
+
+// Grid cell of a value: floor(M * sat((g + alpha) * inv_2alpha)), returned as a float whose BIT
+// PATTERN is that integer (a denormal).  Monotone in g; NaN maps to cell 0.  The same expression is
+// evaluated on the host (cell_of below) when the grid resolution is chosen.
+__device__ __forceinline__ float grid_cell(float g, float alpha, float inv_2alpha, float cell_scale) {
+    return __fmul_rd(mul_sat(__fadd_rn(g, alpha), inv_2alpha), cell_scale);
+}
+
+// [r < T] as 1.0f / 0.0f, where T = rint(p * 2^16) and rf = 2^23 + r.  Both operands of the subtract
+// are integers below 2^24, so the difference is exact; huge or infinite p saturate correctly and a
+// NaN gives 0.
+__device__ __forceinline__ float rounds_up(float p, float rf) {
+    return sub_sat(__fmaf_rn(p, 65536.0f, kMagic), rf);
 }
 
 // Uniform codebook, l_k = -alpha + k * 2 alpha / s (Section 4.1).  Reference form of the decision:
@@ -33,60 +71,104 @@ __device__ __forceinline__ uint32_t rounds_up(float p, uint32_t r16) {
 // x = clip((g + alpha) * inv_step, 0, s), k' = floor x, p' = x - k': the affine map is monotone, so
 // clipping after it gives the same x for |g| <= alpha and 0 / >= s beyond; at x = s this yields
 // k' = s, p' = 0, i.e. the same code s as k = s-1, p >= 1.  NaN becomes 0 (fmaxf drops it).
-__device__ __forceinline__ uint32_t code_uniform(float g, float alpha, float inv_step, float top, uint32_t r16) {
+__device__ __forceinline__ float code_uniform(float g, float alpha, float inv_step, float top, float rf) {
     float x = __fmul_rn(__fadd_rn(g, alpha), inv_step);
     x = fminf(fmaxf(x, 0.0f), top);
-    const float xm = __fadd_rd(x, kMagic);            // mantissa now holds floor(x)
-    const float p = __fsub_rn(x, __fsub_rn(xm, kMagic));
-    return (__float_as_uint(xm) - kMagicBits) + rounds_up(p, r16);
+    const float kf = __fsub_rn(__fadd_rd(x, kMagic), kMagic);   // floor(x), exact
+    return __fadd_rn(kf, rounds_up(__fsub_rn(x, kf), rf));
 }
 
-// General codebook from shared memory: search[] holds l_1 .. l_{s-1} at indices 1 .. s-1 and +inf
-// from index s on, so the branch-free binary search returns k = max{ j <= s-1 : l_j <= t }.
+// General codebook through the lookup grid.  s_grid[c] = (boundary, k_lo): k_lo counts the interior
+// levels in cells below c and `boundary` is the one interior level inside cell c (NaN if none, so that
+// not even +inf compares >= it), so
+// k = k_lo + [g >= boundary] = max{ j <= s-1 : l_j <= g }.  s_cell[k] = (l_k, 1/|Delta_k|).
+// g is not clipped first: beyond +-alpha the same interval is found as for the clipped value, and
+// p >= 1 (or p < 0, or NaN) saturates to the same decision.
+__device__ __forceinline__ float code_grid(float g, float alpha, float inv_2alpha, float cell_scale,
+                                           const char* s_grid, const char* s_cell, float rf) {
+    const float cell8 = __fmul_rn(grid_cell(g, alpha, inv_2alpha, cell_scale), 8.0f);   // bits = 8 * cell
+    const float2 gc = *reinterpret_cast<const float2*>(s_grid + __float_as_uint(cell8));
+    const float kf = __fadd_rn(gc.y, set_ge(g, gc.x));
+    const float k8 = __fmul_rn(kf, __uint_as_float(8u));                                 // bits = 8 * k
+    const float2 c = *reinterpret_cast<const float2*>(s_cell + __float_as_uint(k8));
+    const float p = __fmul_rn(__fsub_rn(g, c.x), c.y);
+    return __fadd_rn(kf, rounds_up(p, rf));
+}
+
+// General codebook by branch-free binary search (used when no grid of at most kMaxGridCells cells
+// separates the levels): search[] holds l_1 .. l_{s-1} at indices 1 .. s-1 and +inf from index s on.
 template <int BITS>
-__device__ __forceinline__ uint32_t code_table(float g, float alpha, const float* search, const float2* cell,
-                                               uint32_t r16) {
+__device__ __forceinline__ float code_binary(float g, float alpha, const float* search, const float2* cell, float rf) {
     const float t = fminf(fmaxf(g, -alpha), alpha);   // NaN -> -alpha
     uint32_t k = 0;
 #pragma unroll
     for (int step = (1 << BITS) >> 1; step > 0; step >>= 1)
         if (t >= search[k + step]) k += step;
-    const float2 c = cell[k];                          // (l_k, 1 / (l_{k+1} - l_k))
+    const float2 c = cell[k];
     const float p = __fmul_rn(__fsub_rn(t, c.x), c.y);
-    return k + rounds_up(p, r16);
+    return __fadd_rn(static_cast<float>(k), rounds_up(p, rf));
 }
 
-template <int BITS, bool NONUNIFORM, bool BF16>
-__global__ void __launch_bounds__(kThreads)
-compress_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
-                const __grid_constant__ CompressArgs args, uint32_t seed_lo, uint32_t seed_hi,
-                uint32_t first_worker, uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_out) {
-    constexpr int L = 1 << BITS;
-    const uint32_t wi = blockIdx.y;
-    const WorkerQ& q = args.q[wi];
-
-    __shared__ float s_search[2 * TQ_MAX_LEVELS];
-    __shared__ float2 s_cell[TQ_MAX_LEVELS];
-    if constexpr (NONUNIFORM) {
-        if (threadIdx.x < 2 * TQ_MAX_LEVELS)
-            s_search[threadIdx.x] = (threadIdx.x >= 1 && threadIdx.x <= L - 2) ? q.levels[threadIdx.x] : __int_as_float(0x7F800000);
-        if (threadIdx.x < L - 1) s_cell[threadIdx.x] = make_float2(q.levels[threadIdx.x], q.inv_width[threadIdx.x]);
-        __syncthreads();
+// Eight float codes (each < 2^BITS) -> their 8*BITS packed bits, LSB first.  The weighted sums are
+// exact in fp32 (below 2^24), so the conversion to integer is exact as well.
+template <int BITS>
+__device__ __forceinline__ uint32_t pack8(const float (&c)[8]) {
+    constexpr float B = static_cast<float>(1 << BITS);
+    if constexpr (BITS <= 3) {
+        float a = c[7];
+#pragma unroll
+        for (int e = 6; e >= 0; --e) a = __fmaf_rn(a, B, c[e]);
+        return __float2uint_rz(a);
+    } else {
+        float lo = c[3], hi = c[7];
+#pragma unroll
+        for (int e = 2; e >= 0; --e) { lo = __fmaf_rn(lo, B, c[e]); hi = __fmaf_rn(hi, B, c[e + 4]); }
+        return __float2uint_rz(lo) + (__float2uint_rz(hi) << 16);
     }
+}
 
-    const uint64_t n_runs = (d + 31) >> 5;
-    const uint64_t run = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x;
-    if (run >= n_runs) return;
+// The ten Philox round keys (key advanced by the Weyl constants), computed once on the host: they
+// depend on the seed only, and sit in the kernel's constant bank instead of registers.
+struct RoundKeys {
+    uint32_t k0[10], k1[10];
+};
 
-    const size_t esz = BF16 ? 2 : 4;
-    const char* row = static_cast<const char*>(grad) + static_cast<uint64_t>(wi) * grad_stride * esz;
+__device__ __forceinline__ void mul_wide(uint32_t a, uint32_t b, uint32_t& hi, uint32_t& lo) {
+    uint64_t p;
+    asm("mul.wide.u32 %0, %1, %2;" : "=l"(p) : "r"(a), "r"(b));
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(p));
+}
+
+// Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11) with the key schedule supplied.
+__device__ __forceinline__ void philox_rounds(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                              const RoundKeys& rk, uint32_t (&out)[4]) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        uint32_t hi0, lo0, hi1, lo1;
+        mul_wide(0xD2511F53u, c0, hi0, lo0);
+        mul_wide(0xCD9E8D57u, c2, hi1, lo1);
+        c0 = hi1 ^ c1 ^ rk.k0[r];
+        c2 = hi0 ^ c3 ^ rk.k1[r];
+        c1 = lo1;
+        c3 = lo0;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+struct RunCtx {
+    float alpha, inv_step, top, inv_2alpha, cell_scale;
+    const char* s_grid; const char* s_cell; const float* s_search;
+};
+
+// One run of 32 elements: load, quantize, pack, store.  TAIL = the last, possibly partial run of a row
+// (element-wise guarded loads, zero padding bits, guarded stores and the row's alignment padding).
+template <int BITS, int SEARCH, bool BF16, bool TAIL>
+__device__ __forceinline__ void compress_run(const char* row, uint32_t* prow, uint64_t run, uint64_t d, uint64_t words_out,
+                                             uint32_t worker, const RoundKeys& rk, const RunCtx& cx) {
+    constexpr size_t esz = BF16 ? 2 : 4;
     const uint64_t j0 = run << 5;
-    const bool full = j0 + 32 <= d;
-    const float alpha = q.alpha, inv_step = q.inv_step, top = q.top;
-    const uint32_t worker = first_worker + wi;
-
     float g[4][8];
-    if (full) {
+    if constexpr (!TAIL) {
 #pragma unroll
         for (int grp = 0; grp < 4; ++grp) load8<BF16>(row + (j0 + 8 * grp) * esz, g[grp]);
     } else {
@@ -99,23 +181,26 @@ compress_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
             }
     }
 
+    const uint32_t blk_lo = static_cast<uint32_t>(j0 >> 3), blk_hi = static_cast<uint32_t>(j0 >> 35);
     uint32_t chunk[4];   // the 8*BITS packed bits of each group
 #pragma unroll
     for (int grp = 0; grp < 4; ++grp) {
-        const uint64_t block = (j0 >> 3) + grp;
         uint32_t rnd[4];
-        philox4x32_10(static_cast<uint32_t>(block), static_cast<uint32_t>(block >> 32), worker, 0u, seed_lo, seed_hi, rnd);
-        uint32_t bitsacc = 0;
+        philox_rounds(blk_lo + grp, blk_hi, worker, 0u, rk, rnd);     // j0 >> 3 is a multiple of 4: no carry
+        float code[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-            const uint32_t r16 = (e & 1) ? (rnd[e >> 1] >> 16) : (rnd[e >> 1] & 0xFFFFu);
-            uint32_t code;
-            if constexpr (NONUNIFORM) code = code_table<BITS>(g[grp][e], alpha, s_search, s_cell, r16);
-            else code = code_uniform(g[grp][e], alpha, inv_step, top, r16);
-            if (!full && j0 + 8 * grp + e >= d) code = 0;     // padding bits are zero
-            bitsacc |= code << (e * BITS);
+            // the element's 16 random bits r as the float 2^23 + r
+            const float rf = __uint_as_float(__byte_perm(rnd[e >> 1], kMagicBits, (e & 1) ? 0x7432u : 0x7410u));
+            if constexpr (SEARCH == kUniform) code[e] = code_uniform(g[grp][e], cx.alpha, cx.inv_step, cx.top, rf);
+            else if constexpr (SEARCH == kGrid)
+                code[e] = code_grid(g[grp][e], cx.alpha, cx.inv_2alpha, cx.cell_scale, cx.s_grid, cx.s_cell, rf);
+            else code[e] = code_binary<BITS>(g[grp][e], cx.alpha, cx.s_search, reinterpret_cast<const float2*>(cx.s_cell), rf);
+            if constexpr (TAIL) {
+                if (j0 + 8 * grp + e >= d) code[e] = 0.0f;     // padding bits are zero
+            }
         }
-        chunk[grp] = bitsacc;
+        chunk[grp] = pack8<BITS>(code);
     }
 
     // four chunks of 8*BITS bits -> BITS words, LSB first
@@ -129,8 +214,8 @@ compress_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
     if constexpr (BITS == 2) { w[0] = chunk[0] | (chunk[1] << 16); w[1] = chunk[2] | (chunk[3] << 16); }
     if constexpr (BITS == 1) { w[0] = chunk[0] | (chunk[1] << 8) | (chunk[2] << 16) | (chunk[3] << 24); }
 
-    uint32_t* dst = packed + static_cast<uint64_t>(wi) * words_stride + run * BITS;
-    if (run + 1 < n_runs) {   // every word of an interior run lies below words_out
+    uint32_t* dst = prow + run * BITS;
+    if constexpr (!TAIL) {   // every word of an interior run lies below words_out
         if constexpr (BITS == 4) *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
         if constexpr (BITS == 3) { dst[0] = w[0]; dst[1] = w[1]; dst[2] = w[2]; }
         if constexpr (BITS == 2) *reinterpret_cast<uint2*>(dst) = make_uint2(w[0], w[1]);
@@ -141,43 +226,142 @@ compress_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
 #pragma unroll
         for (int i = 0; i < BITS; ++i)
             if (first + i < words_out) dst[i] = w[i];
-        uint32_t* rowp = packed + static_cast<uint64_t>(wi) * words_stride;
-        for (uint64_t k = first + BITS; k < words_out; ++k) rowp[k] = 0u;
+        for (uint64_t k = first + BITS; k < words_out; ++k) prow[k] = 0u;
     }
 }
 
-template <int BITS, bool NU, bool BF>
+#ifndef TQ_COMPRESS_MIN_BLOCKS
+#define TQ_COMPRESS_MIN_BLOCKS 4
+#endif
+
+template <int BITS, int SEARCH, bool BF16>
+__global__ void __launch_bounds__(kThreads, TQ_COMPRESS_MIN_BLOCKS)
+compress_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
+                const __grid_constant__ CompressArgs args, const __grid_constant__ RoundKeys rk,
+                uint32_t first_worker, uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_out) {
+    constexpr int L = 1 << BITS;
+    const uint32_t wi = blockIdx.y;
+    const WorkerQ& q = args.q[wi];
+
+    __shared__ __align__(16) float2 s_grid[SEARCH == kGrid ? kMaxGridCells + 1 : 1];
+    __shared__ __align__(16) float2 s_cell[TQ_MAX_LEVELS];
+    __shared__ float s_search[2 * TQ_MAX_LEVELS];
+    if constexpr (SEARCH != kUniform) {
+        if (threadIdx.x < L - 1) s_cell[threadIdx.x] = make_float2(q.levels[threadIdx.x], q.inv_width[threadIdx.x]);
+    }
+    if constexpr (SEARCH == kBinary) {
+        if (threadIdx.x < 2 * TQ_MAX_LEVELS)
+            s_search[threadIdx.x] = (threadIdx.x >= 1 && threadIdx.x <= L - 2) ? q.levels[threadIdx.x] : __int_as_float(0x7F800000);
+    }
+    if constexpr (SEARCH == kGrid) {
+        // cells of the interior levels l_1 .. l_{s-1} (distinct by the host's choice of M)
+        uint32_t lc[L];
+#pragma unroll
+        for (int j = 1; j <= L - 2; ++j)
+            lc[j] = __float_as_uint(grid_cell(q.levels[j], q.alpha, q.inv_2alpha, q.cell_scale));
+        for (uint32_t c = threadIdx.x; c <= q.cells; c += kThreads) {
+            float below = 0.0f, boundary = __int_as_float(0x7FC00000);   // NaN: no value compares >= it
+#pragma unroll
+            for (int j = 1; j <= L - 2; ++j) {
+                if (lc[j] < c) below += 1.0f;
+                if (lc[j] == c) boundary = q.levels[j];
+            }
+            s_grid[c] = make_float2(boundary, below);
+        }
+    }
+    if constexpr (SEARCH != kUniform) __syncthreads();
+
+    constexpr size_t esz = BF16 ? 2 : 4;
+    const char* row = static_cast<const char*>(grad) + static_cast<uint64_t>(wi) * grad_stride * esz;
+    uint32_t* prow = packed + static_cast<uint64_t>(wi) * words_stride;
+    const uint32_t worker = first_worker + wi;
+    const uint64_t n_runs = (d + 31) >> 5;
+    const uint64_t full_runs = d >> 5;
+    const RunCtx cx{q.alpha, q.inv_step, q.top, q.inv_2alpha, q.cell_scale, reinterpret_cast<const char*>(s_grid),
+                    reinterpret_cast<const char*>(s_cell), s_search};
+    const uint64_t stride = static_cast<uint64_t>(gridDim.x) * kThreads;
+
+    uint64_t run = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x;
+    const uint64_t interior = full_runs == n_runs ? n_runs - 1 : full_runs;    // runs that are full AND not the row's last
+    for (; run < interior; run += stride)
+        compress_run<BITS, SEARCH, BF16, false>(row, prow, run, d, words_out, worker, rk, cx);
+    if (run == n_runs - 1)
+        compress_run<BITS, SEARCH, BF16, true>(row, prow, run, d, words_out, worker, rk, cx);
+}
+
+// ---- host side ---------------------------------------------------------------------------------------
+
+// The grid cell of a value, exactly as grid_cell() computes it on the device: every step is a single
+// IEEE operation (u * M is exact for M a power of two), so host and device agree bit for bit.
+static uint32_t cell_of(float g, float alpha, float inv_2alpha, uint32_t cells) {
+    float u = (g + alpha) * inv_2alpha;
+    u = !(u > 0.0f) ? 0.0f : (u > 1.0f ? 1.0f : u);
+    return static_cast<uint32_t>(std::floor(u * static_cast<float>(cells)));
+}
+
+// Smallest power-of-two grid (32 .. 2048 cells) that puts the interior levels in distinct cells; 0 if none.
+static uint32_t choose_cells(const tq_params_t& p, float inv_2alpha) {
+    const int s = static_cast<int>(p.num_levels) - 1;
+    for (uint32_t m = kMinGridCells; m <= static_cast<uint32_t>(kMaxGridCells); m *= 2) {
+        bool distinct = true;
+        for (int j = 2; j <= s - 1 && distinct; ++j)
+            distinct = cell_of(p.levels[j], p.alpha, inv_2alpha, m) > cell_of(p.levels[j - 1], p.alpha, inv_2alpha, m);
+        if (distinct) return m;
+    }
+    return 0;
+}
+
+template <int BITS, int SEARCH, bool BF>
 static cudaError_t launch(const CompressCall& c, const CompressArgs& args, dim3 grid) {
-    compress_kernel<BITS, NU, BF><<<grid, kThreads, 0, c.stream>>>(
-        c.grad, c.d, c.grad_stride, args, static_cast<uint32_t>(c.seed), static_cast<uint32_t>(c.seed >> 32),
-        c.first_worker, c.packed, c.words_stride, c.words_out);
+    RoundKeys rk;
+    uint32_t k0 = static_cast<uint32_t>(c.seed), k1 = static_cast<uint32_t>(c.seed >> 32);
+    for (int r = 0; r < 10; ++r) { rk.k0[r] = k0; rk.k1[r] = k1; k0 += 0x9E3779B9u; k1 += 0xBB67AE85u; }
+    compress_kernel<BITS, SEARCH, BF><<<grid, kThreads, 0, c.stream>>>(
+        c.grad, c.d, c.grad_stride, args, rk, c.first_worker, c.packed, c.words_stride, c.words_out);
     return cudaGetLastError();
 }
 
 template <int BITS>
-static cudaError_t dispatch(const CompressCall& c, const CompressArgs& a, dim3 grid) {
-    if (c.nonuniform) return c.bf16 ? launch<BITS, true, true>(c, a, grid) : launch<BITS, true, false>(c, a, grid);
-    return c.bf16 ? launch<BITS, false, true>(c, a, grid) : launch<BITS, false, false>(c, a, grid);
+static cudaError_t dispatch(const CompressCall& c, const CompressArgs& a, dim3 grid, int search) {
+    if (search == kGrid) return c.bf16 ? launch<BITS, kGrid, true>(c, a, grid) : launch<BITS, kGrid, false>(c, a, grid);
+    if (search == kBinary) return c.bf16 ? launch<BITS, kBinary, true>(c, a, grid) : launch<BITS, kBinary, false>(c, a, grid);
+    return c.bf16 ? launch<BITS, kUniform, true>(c, a, grid) : launch<BITS, kUniform, false>(c, a, grid);
 }
 
 cudaError_t launch_compress(const CompressCall& c) {
     static thread_local CompressArgs args;   // 9 KB: keep it off the stack
+    int search = c.nonuniform ? kGrid : kUniform;
     for (uint32_t i = 0; i < c.n_workers; ++i) {
         const tq_params_t& p = c.params[i];
         WorkerQ& q = args.q[i];
         q.alpha = p.alpha; q.inv_step = p.inv_step; q.top = static_cast<float>(p.num_levels - 1);
+        q.inv_2alpha = 1.0f / (2.0f * p.alpha);
+        q.cells = 0; q.cell_scale = 0.0f;
         for (int k = 0; k < TQ_MAX_LEVELS; ++k) { q.levels[k] = p.levels[k]; q.inv_width[k] = p.inv_width[k]; }
+        if (c.nonuniform) {
+            q.cells = choose_cells(p, q.inv_2alpha);
+            q.cell_scale = std::ldexp(static_cast<float>(q.cells), -149);
+            if (q.cells == 0 || !std::isfinite(q.inv_2alpha)) search = kBinary;
+        }
     }
     const uint64_t n_runs = (c.d + 31) >> 5;
-    const uint64_t blocks = (n_runs + kThreads - 1) / kThreads;
-    if (blocks == 0) return cudaSuccess;
-    if (blocks > 0x7FFFFFFFull) return cudaErrorInvalidConfiguration;
-    const dim3 grid(static_cast<unsigned>(blocks), c.n_workers);
+    const uint64_t tiles = (n_runs + kThreads - 1) / kThreads;
+    if (tiles == 0) return cudaSuccess;
+    // Table modes: persistent blocks (the lookup grid is built once per block), 4 resident blocks per
+    // SM over all workers.  Uniform mode has no per-block set-up, so one block per tile lets the
+    // hardware scheduler balance the tail.
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    uint64_t per_worker = (static_cast<uint64_t>(sms) * TQ_COMPRESS_MIN_BLOCKS + c.n_workers - 1) / c.n_workers;
+    if (search == kUniform || per_worker > tiles) per_worker = tiles;
+    if (per_worker > 0x7FFFFFFFull) per_worker = 0x7FFFFFFFull;
+    if (per_worker < 1) per_worker = 1;
+    const dim3 grid(static_cast<unsigned>(per_worker), c.n_workers);
     switch (c.bits) {
-        case 1: return dispatch<1>(c, args, grid);
-        case 2: return dispatch<2>(c, args, grid);
-        case 3: return dispatch<3>(c, args, grid);
-        default: return dispatch<4>(c, args, grid);
+        case 1: return dispatch<1>(c, args, grid, search);
+        case 2: return dispatch<2>(c, args, grid, search);
+        case 3: return dispatch<3>(c, args, grid, search);
+        default: return dispatch<4>(c, args, grid, search);
     }
 }
 

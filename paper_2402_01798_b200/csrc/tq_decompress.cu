@@ -3,12 +3,11 @@
 // fused in one streaming pass.  fp32 adds happen in worker order, so the result does not depend on
 // the launch shape.
 //
-// Work split: a thread owns the smallest run of elements whose codes fill whole 32-bit words
-// (8 elements for 4 bits, 16 for 2 bits, 32 for 1 bit: one word per worker; 32 elements = 3 words for
-// 3 bits), keeps one fp32 accumulator per element in registers and walks the workers four at a time
-// so that four independent loads are in flight before the dependent lookups start.
-// Codebooks live in shared memory, 16 consecutive words per worker: any set of codes of one worker
-// maps to distinct banks, so lookups are conflict-free.
+// Work split: a thread owns 32 output elements as units whose codes fill whole 32-bit words (see
+// Unit below), keeps one fp32 accumulator per element in registers and walks the workers four at a
+// time so that many independent loads are in flight before the dependent lookups start.
+// Codebooks live in shared memory, 16 consecutive words per worker on a 256-byte pitch: any set of
+// codes of one worker maps to distinct banks, so lookups are conflict-free.
 // HBM traffic per output element: N * bits / 8 bytes read, 4 bytes written.
 #include "tq_device.cuh"
 #include "tq_launch.h"
@@ -25,85 +24,160 @@ __device__ __forceinline__ uint32_t ldg32_stream(const uint32_t* p) {
     return v;
 }
 
+constexpr int kTabStride = 64;   // floats between consecutive workers' codebooks in shared memory (256 bytes)
+
+// A unit is the smallest run of elements whose codes fill whole words: 8 / 16 / 32 elements in one
+// word for 4 / 2 / 1 bits, 32 elements in three words for 3 bits.  A thread owns kUnits units, spaced
+// one block apart, so that every load and every 256-bit store of a warp is contiguous, and keeps
+// kUnits * kElems = 32 accumulators in registers.
 template <int BITS>
 struct Unit {
     static constexpr int kElems = BITS == 4 ? 8 : (BITS == 2 ? 16 : 32);
     static constexpr int kWords = kElems * BITS / 32;
+#ifdef TQ_DECOMPRESS_UNITS4
+    static constexpr int kUnits = TQ_DECOMPRESS_UNITS4 * 8 / kElems > 0 ? TQ_DECOMPRESS_UNITS4 * 8 / kElems : 1;
+#else
+    static constexpr int kUnits = 32 / kElems;
+#endif
 };
 
+// Adds worker `tab`'s dequantized values for the E codes held in w[0 .. W-1] to acc[0 .. E-1].
+// `base` is the byte offset of the worker's codebook in shared memory (a multiple of 256).
 template <int BITS>
-__global__ void __launch_bounds__(kThreads)
+__device__ __forceinline__ void add_unit(float* acc, const uint32_t* w, const char* tab_bytes, uint32_t base) {
+    constexpr int E = Unit<BITS>::kElems, W = Unit<BITS>::kWords;
+    constexpr uint32_t kMask = (1u << BITS) - 1u;
+    if constexpr (W == 1) {
+        // One word holds E = 32 / BITS codes.  The integer pipe is the scarce one here, so the codes
+        // are isolated once per word as bytes already scaled to table offsets (code * 4), and each
+        // lookup offset then costs one byte-permute: plane[j] byte m = 4 * code[m * (8 / BITS) + j];
+        // offset = base with that byte as its low byte.
+        constexpr int kPerByte = 8 / BITS;
+        constexpr uint32_t kPlaneMask = (kMask << 2) * 0x01010101u;
+        uint32_t plane[kPerByte];
+#pragma unroll
+        for (int j = 0; j < kPerByte; ++j) {
+            const int sh = j * BITS - 2;            // bring code j of every byte to bits 2..2+BITS
+            const uint32_t v = sh < 0 ? (w[0] << -sh) : (w[0] >> sh);
+            plane[j] = v & kPlaneMask;
+        }
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            const uint32_t off = __byte_perm(plane[e % kPerByte], base, 0x7650u + (e / kPerByte));
+            acc[e] = __fadd_rn(acc[e], *reinterpret_cast<const float*>(tab_bytes + off));
+        }
+    } else {
+        // 3-bit codes straddle words: funnel-shift the pair of words, mask to a table offset
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            const int pos = e * BITS - 2;
+            const uint32_t lo = w[pos < 0 ? 0 : (pos >> 5)];
+            const uint32_t hi = (pos >= 0 && (pos >> 5) + 1 < W) ? w[(pos >> 5) + 1] : 0u;
+            const uint32_t v = pos < 0 ? (w[0] << 2) : __funnelshift_r(lo, hi, pos & 31);
+            acc[e] = __fadd_rn(acc[e], *reinterpret_cast<const float*>(tab_bytes + ((v & (kMask << 2)) | base)));
+        }
+    }
+}
+
+#ifndef TQ_DECOMPRESS_MIN_BLOCKS
+#define TQ_DECOMPRESS_MIN_BLOCKS 4
+#endif
+
+template <int BITS>
+__global__ void __launch_bounds__(kThreads, TQ_DECOMPRESS_MIN_BLOCKS)
 decompress_kernel(const uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_valid, uint32_t n,
                   uint64_t d, const __grid_constant__ DecompressArgs args, float scale, int divide,
                   float* __restrict__ out) {
-    constexpr int E = Unit<BITS>::kElems, W = Unit<BITS>::kWords;
-    constexpr uint32_t kMask = (1u << BITS) - 1u;
+    constexpr int E = Unit<BITS>::kElems, W = Unit<BITS>::kWords, U = Unit<BITS>::kUnits;
 
-    __shared__ float s_tab[TQ_MAX_WORKERS * TQ_MAX_LEVELS];
+    // Each worker's codebook starts on a 256-byte boundary of shared memory, so a table offset
+    // (code * 4 < 64) can be merged into the worker's base offset by the same byte-permute that
+    // extracts it.  Bank = code: the lookups of one instruction never conflict.
+    __shared__ __align__(256) float s_tab[TQ_MAX_WORKERS * kTabStride];
     for (uint32_t t = threadIdx.x; t < n * TQ_MAX_LEVELS; t += kThreads)
-        s_tab[t] = args.table[t / TQ_MAX_LEVELS][t % TQ_MAX_LEVELS];
+        s_tab[(t / TQ_MAX_LEVELS) * kTabStride + t % TQ_MAX_LEVELS] = args.table[t / TQ_MAX_LEVELS][t % TQ_MAX_LEVELS];
     __syncthreads();
+    const char* tab_bytes = reinterpret_cast<const char*>(s_tab);
 
     const uint64_t n_units = (d + E - 1) / E;
-    const uint64_t u = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x;
-    if (u >= n_units) return;
+    const uint64_t u0 = static_cast<uint64_t>(blockIdx.x) * (kThreads * U) + threadIdx.x;   // unit k of this thread: u0 + k * 256
+    if (u0 >= n_units) return;
 
-    float acc[E];
+    float acc[U][E];
 #pragma unroll
-    for (int e = 0; e < E; ++e) acc[e] = 0.0f;
+    for (int k = 0; k < U; ++k)
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[k][e] = 0.0f;
 
-    const uint64_t w0 = u * W;
-    for (uint32_t i0 = 0; i0 < n; i0 += 4) {
-        uint32_t w[4][W + 1];
+    // interior: all U units exist and all their words lie inside the row
+    const bool interior = u0 + static_cast<uint64_t>(U - 1) * kThreads < n_units &&
+                          (u0 + static_cast<uint64_t>(U - 1) * kThreads) * W + W <= words_valid;
+    const uint32_t* col = packed + u0 * W;
+
+    uint32_t i = 0;
+    if (interior) {
+        for (; i + 4 <= n; i += 4) {          // four workers at a time: 4 * U * W independent loads in flight
+            uint32_t w[4][U][W];
 #pragma unroll
-        for (int b = 0; b < 4; ++b) {
-            const uint32_t* row = packed + static_cast<uint64_t>(i0 + b) * words_stride;
+            for (int b = 0; b < 4; ++b)
 #pragma unroll
-            for (int k = 0; k < W; ++k)
-                w[b][k] = (i0 + b < n && w0 + k < words_valid) ? ldg32_stream(row + w0 + k) : 0u;
-            w[b][W] = 0u;
+                for (int k = 0; k < U; ++k)
+#pragma unroll
+                    for (int x = 0; x < W; ++x)
+                        w[b][k][x] = ldg32_stream(col + static_cast<uint64_t>(i + b) * words_stride + (k * kThreads) * W + x);
+#pragma unroll
+            for (int b = 0; b < 4; ++b)
+#pragma unroll
+                for (int k = 0; k < U; ++k)
+                    add_unit<BITS>(acc[k], w[b][k], tab_bytes + b * (kTabStride * 4), i * (kTabStride * 4));
         }
+    }
+    for (; i < n; ++i) {                       // remaining workers, or every worker of an edge thread
+        uint32_t w[U][W];
 #pragma unroll
-        for (int b = 0; b < 4; ++b) {
-            if (i0 + b < n) {
-                const float* tab = s_tab + (i0 + b) * TQ_MAX_LEVELS;
+        for (int k = 0; k < U; ++k)
 #pragma unroll
-                for (int e = 0; e < E; ++e) {
-                    const int pos = e * BITS;
-                    const uint32_t code = (W == 1) ? ((w[b][0] >> pos) & kMask)
-                                                   : (__funnelshift_r(w[b][pos >> 5], w[b][(pos >> 5) + 1], pos & 31) & kMask);
-                    acc[e] = __fadd_rn(acc[e], tab[code]);
-                }
+            for (int x = 0; x < W; ++x) {
+                const uint64_t idx = (u0 + static_cast<uint64_t>(k) * kThreads) * W + x;
+                w[k][x] = idx < words_valid ? ldg32_stream(packed + static_cast<uint64_t>(i) * words_stride + idx) : 0u;
             }
-        }
+#pragma unroll
+        for (int k = 0; k < U; ++k) add_unit<BITS>(acc[k], w[k], tab_bytes, i * (kTabStride * 4));
     }
 
     // w_i = 1/N: one division by N (for N a power of two the product with 2^-k is the same value)
 #pragma unroll
-    for (int e = 0; e < E; ++e) {
-        if (divide == 1) acc[e] = __fdiv_rn(acc[e], scale);
-        else if (divide == 2) acc[e] = __fmul_rn(acc[e], scale);
-    }
-
-    const uint64_t j0 = u * E;
-    if (j0 + E <= d) {
+    for (int k = 0; k < U; ++k)
 #pragma unroll
-        for (int v = 0; v < E / 8; ++v) {
-            const float o[8] = {acc[8 * v], acc[8 * v + 1], acc[8 * v + 2], acc[8 * v + 3],
-                                acc[8 * v + 4], acc[8 * v + 5], acc[8 * v + 6], acc[8 * v + 7]};
-            stg256(out + j0 + 8 * v, o);
+        for (int e = 0; e < E; ++e) {
+            if (divide == 1) acc[k][e] = __fdiv_rn(acc[k][e], scale);
+            else if (divide == 2) acc[k][e] = __fmul_rn(acc[k][e], scale);
         }
-    } else {
+
 #pragma unroll
-        for (int e = 0; e < E; ++e)
-            if (j0 + e < d) out[j0 + e] = acc[e];
+    for (int k = 0; k < U; ++k) {
+        const uint64_t u = u0 + static_cast<uint64_t>(k) * kThreads;
+        const uint64_t j0 = u * E;
+        if (j0 + E <= d) {
+#pragma unroll
+            for (int v = 0; v < E / 8; ++v) {
+                const float o[8] = {acc[k][8 * v], acc[k][8 * v + 1], acc[k][8 * v + 2], acc[k][8 * v + 3],
+                                    acc[k][8 * v + 4], acc[k][8 * v + 5], acc[k][8 * v + 6], acc[k][8 * v + 7]};
+                stg256(out + j0 + 8 * v, o);
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < E; ++e)
+                if (j0 + e < d) out[j0 + e] = acc[k][e];
+        }
     }
 }
 
 template <int BITS>
 static cudaError_t launch(const DecompressCall& c, const DecompressArgs& args, float scale, int divide) {
     const uint64_t n_units = (c.d + Unit<BITS>::kElems - 1) / Unit<BITS>::kElems;
-    const uint64_t blocks = (n_units + kThreads - 1) / kThreads;
+    const uint64_t per_block = static_cast<uint64_t>(kThreads) * Unit<BITS>::kUnits;
+    const uint64_t blocks = (n_units + per_block - 1) / per_block;
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7FFFFFFFull) return cudaErrorInvalidConfiguration;
     decompress_kernel<BITS><<<static_cast<unsigned>(blocks), kThreads, 0, c.stream>>>(

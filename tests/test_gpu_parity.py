@@ -175,6 +175,33 @@ def test_uniform_table_through_nonuniform_kernel(tq, orc):
     assert np.array_equal(orc.unpack(want, d, 3), ct)
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_compress_caller_codebooks_grid_and_search_paths(tq, orc, dtype):
+    """Caller-supplied codebooks (Section 3.1's general codebook).  Random ones exercise the lookup
+    grid at every resolution; the crowded ones (two levels closer than 1/2048 of the range) force the
+    binary-search path; both must give the oracle's codes."""
+    rng = np.random.default_rng(2024)
+    d = 70_001
+    books = []
+    for L in (4, 8, 16):
+        for trial in range(6):
+            a = float(10.0 ** rng.uniform(-4, 0))
+            inner = np.sort(rng.uniform(-a, a, L - 2) if trial % 2 else a * np.tanh(rng.normal(0, 10.0 ** rng.uniform(-3, 0), L - 2)))
+            lv = np.concatenate([[-a], inner, [a]]).astype(F32)
+            if np.all(np.diff(lv) > 0):
+                books.append(lv)
+        books.append(np.concatenate([[-1.0], np.linspace(0.3, 0.3001, L - 2), [1.0]]).astype(F32))     # crowded
+        books.append(np.concatenate([[-2e-3], np.linspace(-1e-7, 1e-7, L - 2), [2e-3]]).astype(F32))  # crowded at 0
+    for lv in books:
+        p = tq.tq_params_from_levels([float(x) for x in lv])
+        g = heavy_tailed(d, 2, dtype, seed=len(lv), scale=float(lv[-1]) / 8)
+        salt_special_values(g, d, p)
+        got = tq.tq_compress(g, [p, p], seed=77, first_worker=2, d=d).cpu().numpy().view(np.uint32)
+        for i in range(2):
+            want = orc.compress(host_f32(orc, g[i, :d]), to_oracle_params(orc, p), 77, 2 + i)
+            assert np.array_equal(got[i], want), lv
+
+
 # ---------------------------------------------------------------------------- decompress-aggregate
 @pytest.mark.parametrize("bits", [1, 2, 3, 4])
 @pytest.mark.parametrize("n", [1, 2, 3, 5, 8, 16, 33])
