@@ -26,39 +26,64 @@ __device__ __forceinline__ uint32_t ldg32_stream(const uint32_t* p) {
 
 constexpr int kTabStride = 64;   // floats between consecutive workers' codebooks in shared memory (256 bytes)
 
-// A unit is the smallest run of elements whose codes fill whole words: 8 / 16 / 32 elements in one
-// word for 4 / 2 / 1 bits, 32 elements in three words for 3 bits.  A thread owns kUnits units, spaced
-// one block apart, so that every load and every 256-bit store of a warp is contiguous, and keeps
-// kUnits * kElems = 32 accumulators in registers.
+// A unit is a run of elements decoded from one 32-bit "field": 8 / 16 / 32 elements = one packed word
+// for 4 / 2 / 1 bits; for 3 bits 8 elements = 24 bits that start on a byte boundary and are cut out of
+// two neighbouring words.  A thread owns 32 / kElems units, spaced one block apart, so that every
+// load and every 256-bit store of a warp is contiguous, and keeps 32 accumulators in registers.
 template <int BITS>
 struct Unit {
-    static constexpr int kElems = BITS == 4 ? 8 : (BITS == 2 ? 16 : 32);
-    static constexpr int kWords = kElems * BITS / 32;
-#ifdef TQ_DECOMPRESS_UNITS4
-    static constexpr int kUnits = TQ_DECOMPRESS_UNITS4 * 8 / kElems > 0 ? TQ_DECOMPRESS_UNITS4 * 8 / kElems : 1;
-#else
+    static constexpr int kElems = BITS == 2 ? 16 : (BITS == 1 ? 32 : 8);
     static constexpr int kUnits = 32 / kElems;
-#endif
 };
 
-// Adds worker `tab`'s dequantized values for the E codes held in w[0 .. W-1] to acc[0 .. E-1].
-// `base` is the byte offset of the worker's codebook in shared memory (a multiple of 256).
+// The field of unit u of one row, all words known to be inside the row.
 template <int BITS>
-__device__ __forceinline__ void add_unit(float* acc, const uint32_t* w, const char* tab_bytes, uint32_t base) {
-    constexpr int E = Unit<BITS>::kElems, W = Unit<BITS>::kWords;
+__device__ __forceinline__ uint32_t load_field(const uint32_t* row, uint64_t u) {
+    if constexpr (BITS != 3) return ldg32_stream(row + u);
+    else {
+        const uint64_t wi = (3 * u) >> 2;                      // 24 u bits = 3 u bytes into the row
+        const uint32_t sh = (static_cast<uint32_t>(u) * 24u) & 31u;
+        const uint32_t lo = __ldg(row + wi), hi = __ldg(row + wi + 1);   // cached: neighbours share words
+        return __funnelshift_r(lo, hi, sh);
+    }
+}
+// Same with every word checked against the row's length (edge units).
+template <int BITS>
+__device__ __forceinline__ uint32_t load_field_guarded(const uint32_t* row, uint64_t u, uint64_t words_valid) {
+    if constexpr (BITS != 3) return u < words_valid ? ldg32_stream(row + u) : 0u;
+    else {
+        const uint64_t wi = (3 * u) >> 2;
+        const uint32_t sh = (static_cast<uint32_t>(u) * 24u) & 31u;
+        const uint32_t lo = wi < words_valid ? __ldg(row + wi) : 0u;
+        const uint32_t hi = wi + 1 < words_valid ? __ldg(row + wi + 1) : 0u;
+        return __funnelshift_r(lo, hi, sh);
+    }
+}
+// Words of the row a unit needs (for the interior test).
+template <int BITS>
+__device__ __forceinline__ uint64_t last_word_of(uint64_t u) {
+    if constexpr (BITS != 3) return u;
+    else return ((3 * u) >> 2) + 1;
+}
+
+// Adds one worker's dequantized values for the E codes of field f to acc[0 .. E-1].  `tab_bytes + base`
+// is the worker's codebook in shared memory (base a multiple of 256).
+template <int BITS>
+__device__ __forceinline__ void add_unit(float* acc, uint32_t f, const char* tab_bytes, uint32_t base) {
+    constexpr int E = Unit<BITS>::kElems;
     constexpr uint32_t kMask = (1u << BITS) - 1u;
-    if constexpr (W == 1) {
-        // One word holds E = 32 / BITS codes.  The integer pipe is the scarce one here, so the codes
-        // are isolated once per word as bytes already scaled to table offsets (code * 4), and each
-        // lookup offset then costs one byte-permute: plane[j] byte m = 4 * code[m * (8 / BITS) + j];
-        // offset = base with that byte as its low byte.
+    if constexpr (BITS != 3) {
+        // The integer pipe is the scarce one here, so the codes are isolated once per word as bytes
+        // already scaled to table offsets (code * 4), and each lookup offset then costs one
+        // byte-permute: plane[j] byte m = 4 * code[m * (8 / BITS) + j]; offset = base with that byte
+        // as its low byte.
         constexpr int kPerByte = 8 / BITS;
         constexpr uint32_t kPlaneMask = (kMask << 2) * 0x01010101u;
         uint32_t plane[kPerByte];
 #pragma unroll
         for (int j = 0; j < kPerByte; ++j) {
             const int sh = j * BITS - 2;            // bring code j of every byte to bits 2..2+BITS
-            const uint32_t v = sh < 0 ? (w[0] << -sh) : (w[0] >> sh);
+            const uint32_t v = sh < 0 ? (f << -sh) : (f >> sh);
             plane[j] = v & kPlaneMask;
         }
 #pragma unroll
@@ -67,13 +92,11 @@ __device__ __forceinline__ void add_unit(float* acc, const uint32_t* w, const ch
             acc[e] = __fadd_rn(acc[e], *reinterpret_cast<const float*>(tab_bytes + off));
         }
     } else {
-        // 3-bit codes straddle words: funnel-shift the pair of words, mask to a table offset
+        // 3-bit codes do not line up with bytes: shift, then mask-and-merge with the base in one logic op
 #pragma unroll
         for (int e = 0; e < E; ++e) {
-            const int pos = e * BITS - 2;
-            const uint32_t lo = w[pos < 0 ? 0 : (pos >> 5)];
-            const uint32_t hi = (pos >= 0 && (pos >> 5) + 1 < W) ? w[(pos >> 5) + 1] : 0u;
-            const uint32_t v = pos < 0 ? (w[0] << 2) : __funnelshift_r(lo, hi, pos & 31);
+            const int sh = e * BITS - 2;
+            const uint32_t v = sh < 0 ? (f << -sh) : (f >> sh);
             acc[e] = __fadd_rn(acc[e], *reinterpret_cast<const float*>(tab_bytes + ((v & (kMask << 2)) | base)));
         }
     }
@@ -88,7 +111,7 @@ __global__ void __launch_bounds__(kThreads, TQ_DECOMPRESS_MIN_BLOCKS)
 decompress_kernel(const uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_valid, uint32_t n,
                   uint64_t d, const __grid_constant__ DecompressArgs args, float scale, int divide,
                   float* __restrict__ out) {
-    constexpr int E = Unit<BITS>::kElems, W = Unit<BITS>::kWords, U = Unit<BITS>::kUnits;
+    constexpr int E = Unit<BITS>::kElems, U = Unit<BITS>::kUnits;
 
     // Each worker's codebook starts on a 256-byte boundary of shared memory, so a table offset
     // (code * 4 < 64) can be merged into the worker's base offset by the same byte-permute that
@@ -110,39 +133,33 @@ decompress_kernel(const uint32_t* __restrict__ packed, uint64_t words_stride, ui
         for (int e = 0; e < E; ++e) acc[k][e] = 0.0f;
 
     // interior: all U units exist and all their words lie inside the row
-    const bool interior = u0 + static_cast<uint64_t>(U - 1) * kThreads < n_units &&
-                          (u0 + static_cast<uint64_t>(U - 1) * kThreads) * W + W <= words_valid;
-    const uint32_t* col = packed + u0 * W;
+    const uint64_t u_last = u0 + static_cast<uint64_t>(U - 1) * kThreads;
+    const bool interior = u_last < n_units && last_word_of<BITS>(u_last) < words_valid;
 
     uint32_t i = 0;
     if (interior) {
-        for (; i + 4 <= n; i += 4) {          // four workers at a time: 4 * U * W independent loads in flight
-            uint32_t w[4][U][W];
+        for (; i + 4 <= n; i += 4) {          // four workers at a time: 4 * U independent fields in flight
+            uint32_t f[4][U];
 #pragma unroll
             for (int b = 0; b < 4; ++b)
 #pragma unroll
                 for (int k = 0; k < U; ++k)
-#pragma unroll
-                    for (int x = 0; x < W; ++x)
-                        w[b][k][x] = ldg32_stream(col + static_cast<uint64_t>(i + b) * words_stride + (k * kThreads) * W + x);
+                    f[b][k] = load_field<BITS>(packed + static_cast<uint64_t>(i + b) * words_stride, u0 + k * kThreads);
 #pragma unroll
             for (int b = 0; b < 4; ++b)
 #pragma unroll
                 for (int k = 0; k < U; ++k)
-                    add_unit<BITS>(acc[k], w[b][k], tab_bytes + b * (kTabStride * 4), i * (kTabStride * 4));
+                    add_unit<BITS>(acc[k], f[b][k], tab_bytes + b * (kTabStride * 4), i * (kTabStride * 4));
         }
     }
     for (; i < n; ++i) {                       // remaining workers, or every worker of an edge thread
-        uint32_t w[U][W];
+        uint32_t f[U];
 #pragma unroll
         for (int k = 0; k < U; ++k)
+            f[k] = load_field_guarded<BITS>(packed + static_cast<uint64_t>(i) * words_stride,
+                                            u0 + static_cast<uint64_t>(k) * kThreads, words_valid);
 #pragma unroll
-            for (int x = 0; x < W; ++x) {
-                const uint64_t idx = (u0 + static_cast<uint64_t>(k) * kThreads) * W + x;
-                w[k][x] = idx < words_valid ? ldg32_stream(packed + static_cast<uint64_t>(i) * words_stride + idx) : 0u;
-            }
-#pragma unroll
-        for (int k = 0; k < U; ++k) add_unit<BITS>(acc[k], w[k], tab_bytes, i * (kTabStride * 4));
+        for (int k = 0; k < U; ++k) add_unit<BITS>(acc[k], f[k], tab_bytes, i * (kTabStride * 4));
     }
 
     // w_i = 1/N: one division by N (for N a power of two the product with 2^-k is the same value)

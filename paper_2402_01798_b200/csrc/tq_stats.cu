@@ -40,6 +40,12 @@ size_t stats_workspace_bytes(uint32_t n_workers) {
 
 enum Pass { kMoments = 0, kTail = 1, kBoth = 2 };
 
+// Hardware base-2 logarithm (absolute error about 2^-22 for arguments near 1, 2 ulp elsewhere).
+// Subnormal arguments are flushed; only arguments >= 1 (tail elements) are ever used.
+__device__ __forceinline__ float lg2_fast(float x) {
+    float r; asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r;
+}
+
 template <bool BF16, int PASS>
 __global__ void __launch_bounds__(kThreads)
 stats_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride, float g_min_in, float kappa,
@@ -63,29 +69,53 @@ stats_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride, fl
         float g[2][8];
         load8<BF16>(row + (c * kChunk) * esz, g[0]);
         load8<BF16>(row + (c * kChunk + 8) * esz, g[1]);
-        float s_abs = 0.0f, s_sq = 0.0f, s_log = 0.0f;
-        uint32_t c_tail = 0, c_bad = 0;
+        // Fast path: assume every element is finite.  A NaN or Inf (or an overflow of the fp32 partial
+        // sums) shows up as a non-finite partial; the chunk is then redone element by element.
+        float s_abs = 0.0f, s_sq = 0.0f, s_log = 0.0f, c_max = 0.0f;
+        uint32_t c_tail = 0;
 #pragma unroll
         for (int h = 0; h < 2; ++h)
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
                 const float a = fabsf(g[h][e]);
-                const bool ok = a <= 3.402823466e38f;          // false for NaN and Inf
-                const float av = ok ? a : 0.0f;
                 if constexpr (PASS != kTail) {
-                    s_abs += av;
-                    s_sq = fmaf(av, av, s_sq);
-                    max_abs = fmaxf(max_abs, av);
-                    c_bad += ok ? 0u : 1u;
+                    s_abs += a;
+                    s_sq = fmaf(a, a, s_sq);
+                    c_max = fmaxf(c_max, a);        // drops NaN, keeps Inf: only used if the chunk is clean
                 }
                 if constexpr (PASS != kMoments) {
-                    const bool in_tail = tail_on && ok && (a > g_min);
-                    const float lg = __log2f(a * inv_gmin);
+                    const bool in_tail = a > g_min;  // false for NaN, true for Inf (caught below)
+                    const float lg = lg2_fast(a * inv_gmin);
                     s_log += in_tail ? lg : 0.0f;
                     c_tail += in_tail ? 1u : 0u;
                 }
             }
-        sum_abs += s_abs; sum_sq += s_sq; sum_log2 += s_log; n_tail += c_tail; n_bad += c_bad;
+        bool clean = true;
+        if constexpr (PASS != kTail) clean = (s_abs + s_sq) <= 3.402823466e38f;
+        if constexpr (PASS == kTail) clean = s_log <= 3.402823466e38f;
+        else if constexpr (PASS == kBoth) clean = clean && (s_log <= 3.402823466e38f);
+        if (clean) {
+            if constexpr (PASS != kTail) { sum_abs += s_abs; sum_sq += s_sq; max_abs = fmaxf(max_abs, c_max); }
+            if constexpr (PASS != kMoments) {
+                if (tail_on) { sum_log2 += s_log; n_tail += c_tail; }
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float a = fabsf(g[i >> 3][i & 7]);
+                const bool ok = a <= 3.402823466e38f;          // false for NaN and Inf
+                if constexpr (PASS != kTail) {
+                    if (ok) { sum_abs += a; sum_sq += static_cast<double>(a) * a; max_abs = fmaxf(max_abs, a); }
+                    else n_bad += 1;
+                }
+                if constexpr (PASS != kMoments) {
+                    if (tail_on && ok && a > g_min) {
+                        sum_log2 += log2(static_cast<double>(a) * static_cast<double>(inv_gmin));
+                        n_tail += 1;
+                    }
+                }
+            }
+        }
     }
     // the d % 16 leftover elements, taken by the first threads of block 0
     if (blockIdx.x == 0) {
