@@ -33,7 +33,11 @@ constexpr int kTabStride = 64;   // floats between consecutive workers' codebook
 template <int BITS>
 struct Unit {
     static constexpr int kElems = BITS == 2 ? 16 : (BITS == 1 ? 32 : 8);
+#ifdef TQ_DECOMPRESS_ACC
+    static constexpr int kUnits = TQ_DECOMPRESS_ACC / kElems > 0 ? TQ_DECOMPRESS_ACC / kElems : 1;
+#else
     static constexpr int kUnits = 32 / kElems;
+#endif
 };
 
 // The field of unit u of one row, all words known to be inside the row.
@@ -69,7 +73,7 @@ __device__ __forceinline__ uint64_t last_word_of(uint64_t u) {
 // Adds one worker's dequantized values for the E codes of field f to acc[0 .. E-1].  `tab_bytes + base`
 // is the worker's codebook in shared memory (base a multiple of 256).
 template <int BITS>
-__device__ __forceinline__ void add_unit(float* acc, uint32_t f, const char* tab_bytes, uint32_t base) {
+__device__ __forceinline__ void add_unit(f32x2* acc, uint32_t f, const char* tab_bytes, uint32_t base) {
     constexpr int E = Unit<BITS>::kElems;
     constexpr uint32_t kMask = (1u << BITS) - 1u;
     if constexpr (BITS != 3) {
@@ -87,17 +91,20 @@ __device__ __forceinline__ void add_unit(float* acc, uint32_t f, const char* tab
             plane[j] = v & kPlaneMask;
         }
 #pragma unroll
-        for (int e = 0; e < E; ++e) {
-            const uint32_t off = __byte_perm(plane[e % kPerByte], base, 0x7650u + (e / kPerByte));
-            acc[e] = __fadd_rn(acc[e], *reinterpret_cast<const float*>(tab_bytes + off));
+        for (int e = 0; e < E; e += 2) {       // two neighbouring elements per packed add
+            const uint32_t off0 = __byte_perm(plane[e % kPerByte], base, 0x7650u + (e / kPerByte));
+            const uint32_t off1 = __byte_perm(plane[(e + 1) % kPerByte], base, 0x7650u + ((e + 1) / kPerByte));
+            acc[e / 2] = add2(acc[e / 2], pair(*reinterpret_cast<const float*>(tab_bytes + off0),
+                                               *reinterpret_cast<const float*>(tab_bytes + off1)));
         }
     } else {
         // 3-bit codes do not line up with bytes: shift, then mask-and-merge with the base in one logic op
 #pragma unroll
-        for (int e = 0; e < E; ++e) {
-            const int sh = e * BITS - 2;
-            const uint32_t v = sh < 0 ? (f << -sh) : (f >> sh);
-            acc[e] = __fadd_rn(acc[e], *reinterpret_cast<const float*>(tab_bytes + ((v & (kMask << 2)) | base)));
+        for (int e = 0; e < E; e += 2) {
+            const int sh0 = e * BITS - 2, sh1 = (e + 1) * BITS - 2;
+            const uint32_t v0 = sh0 < 0 ? (f << -sh0) : (f >> sh0), v1 = f >> sh1;
+            acc[e / 2] = add2(acc[e / 2], pair(*reinterpret_cast<const float*>(tab_bytes + ((v0 & (kMask << 2)) | base)),
+                                               *reinterpret_cast<const float*>(tab_bytes + ((v1 & (kMask << 2)) | base))));
         }
     }
 }
@@ -126,11 +133,11 @@ decompress_kernel(const uint32_t* __restrict__ packed, uint64_t words_stride, ui
     const uint64_t u0 = static_cast<uint64_t>(blockIdx.x) * (kThreads * U) + threadIdx.x;   // unit k of this thread: u0 + k * 256
     if (u0 >= n_units) return;
 
-    float acc[U][E];
+    f32x2 acc[U][E / 2];          // fp32 accumulators, two per 64-bit register pair
 #pragma unroll
     for (int k = 0; k < U; ++k)
 #pragma unroll
-        for (int e = 0; e < E; ++e) acc[k][e] = 0.0f;
+        for (int e = 0; e < E / 2; ++e) acc[k][e] = both(0.0f);
 
     // interior: all U units exist and all their words lie inside the row
     const uint64_t u_last = u0 + static_cast<uint64_t>(U - 1) * kThreads;
@@ -164,28 +171,28 @@ decompress_kernel(const uint32_t* __restrict__ packed, uint64_t words_stride, ui
 
     // w_i = 1/N: one division by N (for N a power of two the product with 2^-k is the same value)
 #pragma unroll
-    for (int k = 0; k < U; ++k)
+    for (int k = 0; k < U; ++k) {
+        float o[E];
+#pragma unroll
+        for (int e = 0; e < E / 2; ++e) unpair(acc[k][e], o[2 * e], o[2 * e + 1]);
 #pragma unroll
         for (int e = 0; e < E; ++e) {
-            if (divide == 1) acc[k][e] = __fdiv_rn(acc[k][e], scale);
-            else if (divide == 2) acc[k][e] = __fmul_rn(acc[k][e], scale);
+            if (divide == 1) o[e] = __fdiv_rn(o[e], scale);
+            else if (divide == 2) o[e] = __fmul_rn(o[e], scale);
         }
-
-#pragma unroll
-    for (int k = 0; k < U; ++k) {
         const uint64_t u = u0 + static_cast<uint64_t>(k) * kThreads;
         const uint64_t j0 = u * E;
         if (j0 + E <= d) {
 #pragma unroll
             for (int v = 0; v < E / 8; ++v) {
-                const float o[8] = {acc[k][8 * v], acc[k][8 * v + 1], acc[k][8 * v + 2], acc[k][8 * v + 3],
-                                    acc[k][8 * v + 4], acc[k][8 * v + 5], acc[k][8 * v + 6], acc[k][8 * v + 7]};
-                stg256(out + j0 + 8 * v, o);
+                const float o8[8] = {o[8 * v], o[8 * v + 1], o[8 * v + 2], o[8 * v + 3],
+                                     o[8 * v + 4], o[8 * v + 5], o[8 * v + 6], o[8 * v + 7]};
+                stg256(out + j0 + 8 * v, o8);
             }
         } else {
 #pragma unroll
             for (int e = 0; e < E; ++e)
-                if (j0 + e < d) out[j0 + e] = acc[k][e];
+                if (j0 + e < d) out[j0 + e] = o[e];
         }
     }
 }
