@@ -120,8 +120,13 @@ def _grad_layout(grad: torch.Tensor, d: Optional[int]):
     return n, (width if d is None else d), (grad.stride(0) if n > 1 else width)
 
 
-def _params_array(params: Sequence[Params]):
+def params_array(params: Sequence[Params]):
+    """A contiguous tq_params_t[N] for tq_compress / tq_decompress_aggregate (build once, pass many times)."""
     return (Params * len(params))(*params)
+
+
+def _params_array(params):
+    return params if isinstance(params, C.Array) else params_array(params)
 
 
 # ------------------------------------------------------------------------------------------------
