@@ -30,6 +30,9 @@ if ROOT not in sys.path:
 
 METRIC = "compress & decompress-aggregate GB/s of fp32 gradient, % of B200 HBM peak"
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised in
+# profiles/compress_kernel_resnet50-25.6M.md (valid for the kernel as it stands; None elsewhere)
+NCU_DRAM_BYTES = {("resnet50-25.6M", "tq_compress"): 1_843_500_000}
 
 
 def hbm_peak():
@@ -276,9 +279,10 @@ def main():
     kernels["tq_decompress_aggregate"]["cold_l2_frac_of_hbm_peak"] = kb / (t_cold * 1e-3) / 1e9 / peak
     del flush
 
-    dom = "tq_compress"
+    dom = "tq_compress"      # the single kernel with the largest share of the round (see profiles/launch_list_*)
     roofline = {"kernel": dom, "bound": "hbm", "achieved": kernels[dom]["gbs"], "peak": peak, "peak_source": peak_kind,
-                "unit": "GB/s", "frac": kernels[dom]["gbs"] / peak, "traffic": None}
+                "unit": "GB/s", "frac": kernels[dom]["gbs"] / peak, "algorithmic_bytes": alg[dom][0],
+                "traffic": NCU_DRAM_BYTES.get((w.name, dom))}
 
     # end to end through the public API with HOST buffers: H2D of every worker's gradient, the round,
     # D2H of the aggregated update, all inside the timed region
