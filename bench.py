@@ -96,6 +96,28 @@ class ClockSampler:
         return out
 
 
+def replica_workload(w, rank: int):
+    """The workload rank `rank` runs: the same shapes with its own seeds (a replica, not a shard)."""
+    from dataclasses import replace
+    return replace(w, base_seed=w.base_seed + 1000 * rank)
+
+
+def max_over_ranks(ms: float, world: int, device="cpu") -> float:
+    """Slowest rank's time: the only cross-rank exchange of the benchmark (timing, not data)."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gbs(world: int, bytes_per_rank: int, ms: float) -> float:
+    """Aggregate throughput of all ranks: every rank processes bytes_per_rank in the slowest rank's time."""
+    return world * bytes_per_rank / (ms * 1e-3) / 1e9
+
+
 def cpu_oracle_round(w, sample_d: int, seed: int = 0):
     """One round of the path by the CPU oracle on `sample_d` elements per worker.  Returns seconds."""
     import numpy as np
@@ -189,8 +211,7 @@ def main():
     N, d, bits = w.n_workers, w.d, w.bits
 
     # inputs resident in HBM (rank r uses its own seeds: a replica, not a shard)
-    from dataclasses import replace
-    wr = replace(w, base_seed=w.base_seed + 1000 * rank)
+    wr = replica_workload(w, rank)
     g, stride = inputs.make_worker_gradients(wr, dev)
     words = tq.tq_packed_words(d, bits)
     packed = torch.empty((N, words), dtype=torch.int32, device=dev)
@@ -240,13 +261,10 @@ def main():
     clocks = sampler.stop()
     total_ms = t_start.elapsed_time(t_end)
 
-    if world > 1:
-        tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        torch.distributed.all_reduce(tt, op=torch.distributed.ReduceOp.MAX)
-        total_ms = float(tt.item())
+    total_ms = max_over_ranks(total_ms, world, dev)
     ms_per_step = total_ms / args.steps
     in_bytes = N * d * esz
-    value = world * in_bytes / (ms_per_step * 1e-3) / 1e9
+    value = whole_job_gbs(world, in_bytes, ms_per_step)
 
     # per-kernel durations inside the timed region (CUDA events on the launching stream)
     t_stats = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)       # two launches
@@ -314,12 +332,8 @@ def main():
         b.record()
         barrier()
         ems = a.elapsed_time(b)
-        if world > 1:
-            tt = torch.tensor([ems], device=dev, dtype=torch.float64)
-            torch.distributed.all_reduce(tt, op=torch.distributed.ReduceOp.MAX)
-            ems = float(tt.item())
-        ems /= e2e_steps
-        e2e = {"value": world * in_bytes / (ems * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": ems,
+        ems = max_over_ranks(ems, world, dev) / e2e_steps
+        e2e = {"value": whole_job_gbs(world, in_bytes, ems), "unit": "GB/s", "ms_per_step": ems,
                "h2d_bytes_per_step": int(N * stride * esz), "d2h_bytes_per_step": int(4 * d + 64 * N)}
         del host_g, host_out, g2
 
