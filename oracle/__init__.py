@@ -73,7 +73,8 @@ _lib = None
 def lib() -> C.CDLL:
     global _lib
     if _lib is None:
-        L = C.CDLL(build())
+        # TQ_ORACLE_LIB: load another build of the oracle (the mutation test plants mistakes this way)
+        L = C.CDLL(os.environ.get("TQ_ORACLE_LIB") or build())
         u32, u64, f32, f64, i32 = C.c_uint32, C.c_uint64, C.c_float, C.c_double, C.c_int
         P = C.POINTER
         L.orc_philox4x32_10.argtypes = [P(u32), P(u32), P(u32)]
