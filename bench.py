@@ -181,6 +181,8 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=2, help="index into the five workloads (default: 25.6M x 16)")
+    ap.add_argument("--variant", type=int, default=None,
+                    help="with --config 3: index 0..11 into the bf16 sweep (gamma x mode x levels)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -189,6 +191,8 @@ def main():
 
     from paper_2402_01798_b200 import inputs
     w = inputs.WORKLOADS[args.config]
+    if args.config == 3 and args.variant is not None:
+        w = inputs.CONFIG4_SWEEP[args.variant]
     if args.impl == "reference":
         run_reference(args, w)
         return

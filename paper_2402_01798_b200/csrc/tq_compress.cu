@@ -66,33 +66,49 @@ __device__ __forceinline__ float rounds_up(float p, float rf) {
     return sub_sat(__fmaf_rn(p, 65536.0f, kMagic), rf);
 }
 
-// Uniform codebook, l_k = -alpha + k * 2 alpha / s (Section 4.1).  Reference form of the decision:
-// t = clip(g), x = (t + alpha) * inv_step, k = min(floor x, s-1), p = x - k.  Computed here as
-// x = clip((g + alpha) * inv_step, 0, s), k' = floor x, p' = x - k': the affine map is monotone, so
-// clipping after it gives the same x for |g| <= alpha and 0 / >= s beyond; at x = s this yields
-// k' = s, p' = 0, i.e. the same code s as k = s-1, p >= 1.  NaN becomes 0 (fmaxf drops it).
-__device__ __forceinline__ float code_uniform(float g, float alpha, float inv_step, float top, float rf) {
-    float x = __fmul_rn(__fadd_rn(g, alpha), inv_step);
-    x = fminf(fmaxf(x, 0.0f), top);
-    const float kf = __fsub_rn(__fadd_rd(x, kMagic), kMagic);   // floor(x), exact
-    return __fadd_rn(kf, rounds_up(__fsub_rn(x, kf), rf));
+// Uniform codebook, l_k = -alpha + k * 2 alpha / s (Section 4.1), two elements at a time.  Reference
+// form of the decision: t = clip(g), x = (t + alpha) * inv_step, k = min(floor x, s-1), p = x - k.
+// Computed here as x = clip((g + alpha) * inv_step, 0, s), k' = floor x, p' = x - k': the affine map is
+// monotone, so clipping after it gives the same x for |g| <= alpha and 0 / >= s beyond; at x = s this
+// yields k' = s, p' = 0, i.e. the same code s as k = s-1, p >= 1.  NaN becomes 0 (fmaxf drops it).
+__device__ __forceinline__ f32x2 code_uniform2(float g0, float g1, f32x2 alpha2, f32x2 inv_step2, float top,
+                                               float rf0, float rf1) {
+    float x0, x1;
+    unpair(mul2(add2(pair(g0, g1), alpha2), inv_step2), x0, x1);
+    const f32x2 x = pair(fminf(fmaxf(x0, 0.0f), top), fminf(fmaxf(x1, 0.0f), top));
+    const f32x2 magic2 = both(kMagic);
+    const f32x2 kf = sub2(add2_rd(x, magic2), magic2);                       // floor(x), exact
+    float pm0, pm1;
+    unpair(fma2(sub2(x, kf), both(65536.0f), magic2), pm0, pm1);            // 2^23 + rint(p * 2^16)
+    return add2(kf, pair(sub_sat(pm0, rf0), sub_sat(pm1, rf1)));
 }
 
-// General codebook through the lookup grid.  s_grid[c] = (boundary, k_lo): k_lo counts the interior
-// levels in cells below c and `boundary` is the one interior level inside cell c (NaN if none, so that
-// not even +inf compares >= it), so
+// General codebook through the lookup grid, two elements at a time.  s_grid[c] = (boundary, k_lo): k_lo
+// counts the interior levels in cells below c and `boundary` is the one interior level inside cell c
+// (NaN if none, so that not even +inf compares >= it), so
 // k = k_lo + [g >= boundary] = max{ j <= s-1 : l_j <= g }.  s_cell[k] = (l_k, 1/|Delta_k|).
 // g is not clipped first: beyond +-alpha the same interval is found as for the clipped value, and
 // p >= 1 (or p < 0, or NaN) saturates to the same decision.
-__device__ __forceinline__ float code_grid(float g, float alpha, float inv_2alpha, float cell_scale,
-                                           const char* s_grid, const char* s_cell, float rf) {
-    const float cell8 = __fmul_rn(grid_cell(g, alpha, inv_2alpha, cell_scale), 8.0f);   // bits = 8 * cell
-    const float2 gc = *reinterpret_cast<const float2*>(s_grid + __float_as_uint(cell8));
-    const float kf = __fadd_rn(gc.y, set_ge(g, gc.x));
-    const float k8 = __fmul_rn(kf, __uint_as_float(8u));                                 // bits = 8 * k
-    const float2 c = *reinterpret_cast<const float2*>(s_cell + __float_as_uint(k8));
-    const float p = __fmul_rn(__fsub_rn(g, c.x), c.y);
-    return __fadd_rn(kf, rounds_up(p, rf));
+__device__ __forceinline__ f32x2 code_grid2(float g0, float g1, f32x2 alpha2, float inv_2alpha, f32x2 cell_scale2,
+                                            const char* s_grid, const char* s_cell, float rf0, float rf1) {
+    const f32x2 g = pair(g0, g1);
+    float s0, s1;
+    unpair(add2(g, alpha2), s0, s1);
+    // cell = floor(M * sat((g + alpha) * inv_2alpha)) as a denormal whose bit pattern is the integer; * 8 = byte offset
+    const f32x2 cell8 = mul2(mul2_rd(pair(mul_sat(s0, inv_2alpha), mul_sat(s1, inv_2alpha)), cell_scale2), both(8.0f));
+    float c0, c1;
+    unpair(cell8, c0, c1);
+    const float2 gc0 = *reinterpret_cast<const float2*>(s_grid + __float_as_uint(c0));
+    const float2 gc1 = *reinterpret_cast<const float2*>(s_grid + __float_as_uint(c1));
+    const f32x2 kf = add2(pair(gc0.y, gc1.y), pair(set_ge(g0, gc0.x), set_ge(g1, gc1.x)));
+    float k0, k1;
+    unpair(mul2(kf, both(__uint_as_float(8u))), k0, k1);                     // bits = 8 * k
+    const float2 q0 = *reinterpret_cast<const float2*>(s_cell + __float_as_uint(k0));
+    const float2 q1 = *reinterpret_cast<const float2*>(s_cell + __float_as_uint(k1));
+    const f32x2 p = mul2(sub2(g, pair(q0.x, q1.x)), pair(q0.y, q1.y));
+    float pm0, pm1;
+    unpair(fma2(p, both(65536.0f), both(kMagic)), pm0, pm1);
+    return add2(kf, pair(sub_sat(pm0, rf0), sub_sat(pm1, rf1)));
 }
 
 // General codebook by branch-free binary search (used when no grid of at most kMaxGridCells cells
@@ -109,21 +125,23 @@ __device__ __forceinline__ float code_binary(float g, float alpha, const float* 
     return __fadd_rn(static_cast<float>(k), rounds_up(p, rf));
 }
 
-// Eight float codes (each < 2^BITS) -> their 8*BITS packed bits, LSB first.  The weighted sums are
-// exact in fp32 (below 2^24), so the conversion to integer is exact as well.
+// Four pairs of float codes (elements 0..7 of a group, each code < 2^BITS) -> their 8*BITS packed
+// bits, LSB first.  Every partial sum is an integer below 2^24, so the fp32 arithmetic is exact.
 template <int BITS>
-__device__ __forceinline__ uint32_t pack8(const float (&c)[8]) {
-    constexpr float B = static_cast<float>(1 << BITS);
+__device__ __forceinline__ uint32_t pack8(const f32x2 (&c)[4]) {
+    constexpr float B = static_cast<float>(1 << BITS), B2 = B * B;
     if constexpr (BITS <= 3) {
-        float a = c[7];
-#pragma unroll
-        for (int e = 6; e >= 0; --e) a = __fmaf_rn(a, B, c[e]);
-        return __float2uint_rz(a);
+        f32x2 a = fma2(c[3], both(B2), c[2]);
+        a = fma2(a, both(B2), c[1]);
+        a = fma2(a, both(B2), c[0]);
+        float ev, od;
+        unpair(a, ev, od);
+        return __float2uint_rz(__fmaf_rn(od, B, ev));
     } else {
-        float lo = c[3], hi = c[7];
-#pragma unroll
-        for (int e = 2; e >= 0; --e) { lo = __fmaf_rn(lo, B, c[e]); hi = __fmaf_rn(hi, B, c[e + 4]); }
-        return __float2uint_rz(lo) + (__float2uint_rz(hi) << 16);
+        float e0, o0, e1, o1;
+        unpair(fma2(c[1], both(B2), c[0]), e0, o0);       // elements 0..3: 16 bits
+        unpair(fma2(c[3], both(B2), c[2]), e1, o1);       // elements 4..7: 16 bits
+        return __float2uint_rz(__fmaf_rn(o0, B, e0)) + (__float2uint_rz(__fmaf_rn(o1, B, e1)) << 16);
     }
 }
 
@@ -160,6 +178,11 @@ struct RunCtx {
     const char* s_grid; const char* s_cell; const float* s_search;
 };
 
+// the 16 random bits of slot e of a Philox block, as the float 2^23 + r
+__device__ __forceinline__ float slot_as_float(const uint32_t (&rnd)[4], int e) {
+    return __uint_as_float(__byte_perm(rnd[e >> 1], kMagicBits, (e & 1) ? 0x7432u : 0x7410u));
+}
+
 // One run of 32 elements: load, quantize, pack, store.  TAIL = the last, possibly partial run of a row
 // (element-wise guarded loads, zero padding bits, guarded stores and the row's alignment padding).
 template <int BITS, int SEARCH, bool BF16, bool TAIL>
@@ -167,37 +190,44 @@ __device__ __forceinline__ void compress_run(const char* row, uint32_t* prow, ui
                                              uint32_t worker, const RoundKeys& rk, const RunCtx& cx) {
     constexpr size_t esz = BF16 ? 2 : 4;
     const uint64_t j0 = run << 5;
-    float g[4][8];
+    Raw8<BF16> g[4];
     if constexpr (!TAIL) {
 #pragma unroll
-        for (int grp = 0; grp < 4; ++grp) load8<BF16>(row + (j0 + 8 * grp) * esz, g[grp]);
+        for (int grp = 0; grp < 4; ++grp) load8_raw<BF16>(row + (j0 + 8 * grp) * esz, g[grp]);
     } else {
 #pragma unroll
         for (int grp = 0; grp < 4; ++grp)
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
                 const uint64_t j = j0 + 8 * grp + e;
-                g[grp][e] = j < d ? load1<BF16>(row, j) : 0.0f;
+                set_elem<BF16>(g[grp], e, j < d ? load1<BF16>(row, j) : 0.0f);
             }
     }
 
     const uint32_t blk_lo = static_cast<uint32_t>(j0 >> 3), blk_hi = static_cast<uint32_t>(j0 >> 35);
+    const f32x2 alpha2 = both(cx.alpha), inv_step2 = both(cx.inv_step), cell_scale2 = both(cx.cell_scale);
     uint32_t chunk[4];   // the 8*BITS packed bits of each group
 #pragma unroll
     for (int grp = 0; grp < 4; ++grp) {
         uint32_t rnd[4];
         philox_rounds(blk_lo + grp, blk_hi, worker, 0u, rk, rnd);     // j0 >> 3 is a multiple of 4: no carry
-        float code[8];
+        f32x2 code[4];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            // the element's 16 random bits r as the float 2^23 + r
-            const float rf = __uint_as_float(__byte_perm(rnd[e >> 1], kMagicBits, (e & 1) ? 0x7432u : 0x7410u));
-            if constexpr (SEARCH == kUniform) code[e] = code_uniform(g[grp][e], cx.alpha, cx.inv_step, cx.top, rf);
+        for (int h = 0; h < 4; ++h) {            // elements 2h, 2h+1 of the group
+            const int e = 2 * h;
+            const float rf0 = slot_as_float(rnd, e), rf1 = slot_as_float(rnd, e + 1);
+            const float g0 = elem<BF16>(g[grp], e), g1 = elem<BF16>(g[grp], e + 1);
+            if constexpr (SEARCH == kUniform) code[h] = code_uniform2(g0, g1, alpha2, inv_step2, cx.top, rf0, rf1);
             else if constexpr (SEARCH == kGrid)
-                code[e] = code_grid(g[grp][e], cx.alpha, cx.inv_2alpha, cx.cell_scale, cx.s_grid, cx.s_cell, rf);
-            else code[e] = code_binary<BITS>(g[grp][e], cx.alpha, cx.s_search, reinterpret_cast<const float2*>(cx.s_cell), rf);
-            if constexpr (TAIL) {
-                if (j0 + 8 * grp + e >= d) code[e] = 0.0f;     // padding bits are zero
+                code[h] = code_grid2(g0, g1, alpha2, cx.inv_2alpha, cell_scale2, cx.s_grid, cx.s_cell, rf0, rf1);
+            else code[h] = pair(code_binary<BITS>(g0, cx.alpha, cx.s_search, reinterpret_cast<const float2*>(cx.s_cell), rf0),
+                                code_binary<BITS>(g1, cx.alpha, cx.s_search, reinterpret_cast<const float2*>(cx.s_cell), rf1));
+            if constexpr (TAIL) {                 // padding bits are zero
+                float c0, c1;
+                unpair(code[h], c0, c1);
+                if (j0 + 8 * grp + e >= d) c0 = 0.0f;
+                if (j0 + 8 * grp + e + 1 >= d) c1 = 0.0f;
+                code[h] = pair(c0, c1);
             }
         }
         chunk[grp] = pack8<BITS>(code);

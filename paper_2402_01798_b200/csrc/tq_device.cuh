@@ -45,6 +45,30 @@ __device__ __forceinline__ void load8(const void* p, float (&g)[8]) {
     }
 }
 
+// Eight consecutive gradient elements kept as loaded (fp32: 8 words; bf16: 4 words of two), decoded
+// on use.  Keeping bf16 packed halves the registers a loaded group occupies.
+template <bool BF16>
+struct Raw8 {
+    uint32_t v[BF16 ? 4 : 8];
+};
+template <bool BF16>
+__device__ __forceinline__ void load8_raw(const void* p, Raw8<BF16>& r) {
+    if constexpr (!BF16) ldg256_stream(p, r.v);
+    else asm volatile("ld.global.nc.L1::no_allocate.v4.b32 {%0,%1,%2,%3}, [%4];"
+                      : "=r"(r.v[0]), "=r"(r.v[1]), "=r"(r.v[2]), "=r"(r.v[3]) : "l"(p));
+}
+template <bool BF16>
+__device__ __forceinline__ float elem(const Raw8<BF16>& r, int e) {
+    if constexpr (!BF16) return __uint_as_float(r.v[e]);
+    else return __uint_as_float((e & 1) ? (r.v[e >> 1] & 0xFFFF0000u) : (r.v[e >> 1] << 16));
+}
+template <bool BF16>
+__device__ __forceinline__ void set_elem(Raw8<BF16>& r, int e, float x) {   // fp32 bits, or an exact bf16 value
+    if constexpr (!BF16) r.v[e] = __float_as_uint(x);
+    else r.v[e >> 1] = (e & 1) ? ((r.v[e >> 1] & 0x0000FFFFu) | (__float_as_uint(x) & 0xFFFF0000u))
+                               : ((r.v[e >> 1] & 0xFFFF0000u) | (__float_as_uint(x) >> 16));
+}
+
 // One element, any alignment (ragged tails).
 template <bool BF16>
 __device__ __forceinline__ float load1(const void* base, uint64_t j) {
