@@ -231,9 +231,7 @@ def main():
         if ev: ev[1].record()
         stats_pin.copy_(stats_dev, non_blocking=True)
         stream.synchronize()                                   # the only host sync of a round
-        raw = stats_pin.numpy().tobytes()
-        ps = tq.params_array([tq.tq_params(tq.Stats.from_buffer_copy(raw[i * 64:(i + 1) * 64]), w.num_levels, mode, w.gamma)
-                              for i in range(N)])
+        ps = tq.tq_params_batch(stats_pin, N, w.num_levels, mode, w.gamma)
         if ev: ev[2].record()
         tq.tq_compress(g, ps, seed=1234, d=d, packed=packed)
         if ev: ev[3].record()
@@ -321,9 +319,7 @@ def main():
             tq.tq_stats(g2, d, stats_dev=stats_dev, workspace=ws)
             stats_pin.copy_(stats_dev, non_blocking=True)
             stream.synchronize()
-            raw = stats_pin.numpy().tobytes()
-            pp = tq.params_array([tq.tq_params(tq.Stats.from_buffer_copy(raw[i * 64:(i + 1) * 64]), w.num_levels, mode, w.gamma)
-                                  for i in range(N)])
+            pp = tq.tq_params_batch(stats_pin, N, w.num_levels, mode, w.gamma)
             tq.tq_compress(g2, pp, seed=1234, d=d, packed=packed)
             tq.tq_decompress_aggregate(packed, d, pp, out=out)
             host_out.copy_(out, non_blocking=True)

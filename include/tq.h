@@ -160,6 +160,11 @@ tq_status tq_stats_static(const void* grad_dev, tq_dtype dtype, uint64_t d, uint
 tq_status tq_params(const tq_stats_t* stats_host, uint32_t num_levels, tq_mode mode, double gamma,
                     tq_alpha_rule alpha_rule, double alpha_user, tq_params_t* out_host);
 
+/* tq_params for n workers in one call: stats_host[n] -> out_host[n], same arguments for all.
+ * Stops at the first failing worker and returns its status. */
+tq_status tq_params_batch(const tq_stats_t* stats_host, uint32_t n_workers, uint32_t num_levels, tq_mode mode,
+                          double gamma, tq_alpha_rule alpha_rule, double alpha_user, tq_params_t* out_host);
+
 /* Quantizer for a caller-supplied codebook (any strictly increasing levels with
  * levels[0] = -levels[L-1]; Section 3.1's general codebook).  Fills inv_width / inv_step. */
 tq_status tq_params_from_levels(const float* levels_host, uint32_t num_levels, tq_mode mode,

@@ -25,7 +25,7 @@ UNIFORM, NONUNIFORM = 0, 1
 ALPHA_CLOSED, ALPHA_FIXED_POINT, ALPHA_USER = 0, 1, 2
 FLAG_ALPHA_CAPPED, FLAG_ALPHA_AT_GMIN, FLAG_GAMMA_FROM_MLE = 1, 2, 4
 
-EXPORTS = ("tq_packed_words", "tq_stats_workspace_bytes", "tq_stats", "tq_stats_static", "tq_params", "tq_params_from_levels",
+EXPORTS = ("tq_packed_words", "tq_stats_workspace_bytes", "tq_stats", "tq_stats_static", "tq_params", "tq_params_batch", "tq_params_from_levels",
            "tq_compress", "tq_decompress_aggregate", "tq_strerror", "tq_last_cuda_error", "tq_kernel_launches")
 
 
@@ -72,6 +72,8 @@ def lib() -> C.CDLL:
         L.tq_stats_static.argtypes = [vp, C.c_int, u64, u64, u32, f32, f32, vp, vp]; L.tq_stats_static.restype = C.c_int
         L.tq_params.argtypes = [C.POINTER(Stats), u32, C.c_int, f64, C.c_int, f64, C.POINTER(Params)]
         L.tq_params.restype = C.c_int
+        L.tq_params_batch.argtypes = [vp, u32, u32, C.c_int, f64, C.c_int, f64, vp]
+        L.tq_params_batch.restype = C.c_int
         L.tq_params_from_levels.argtypes = [C.POINTER(f32), u32, C.c_int, C.POINTER(Params)]
         L.tq_params_from_levels.restype = C.c_int
         L.tq_compress.argtypes = [vp, C.c_int, u64, u64, u32, C.POINTER(Params), u64, u32, vp, sz, vp]
@@ -176,6 +178,22 @@ def tq_params(stats: Stats, num_levels: int, mode: int, gamma: float = math.nan,
     p = Params()
     _check(lib().tq_params(C.byref(stats), num_levels, mode, gamma, alpha_rule, alpha_user, C.byref(p)), "tq_params")
     return p
+
+
+def tq_params_batch(stats_raw, n_workers: int, num_levels: int, mode: int, gamma: float = math.nan,
+                    alpha_rule: int = ALPHA_FIXED_POINT, alpha_user: float = 0.0):
+    """tq_params for n workers at once.  ``stats_raw``: the n 64-byte records as bytes, a ctypes array of
+    Stats, or a pinned CPU uint8 tensor (used in place).  Returns a ctypes tq_params_t[n] array."""
+    out = (Params * n_workers)()
+    if isinstance(stats_raw, torch.Tensor):
+        src = C.c_void_p(stats_raw.data_ptr())
+    elif isinstance(stats_raw, (bytes, bytearray)):
+        src = C.cast(C.create_string_buffer(bytes(stats_raw), len(stats_raw)), C.c_void_p)
+    else:
+        src = C.cast(stats_raw, C.c_void_p)
+    _check(lib().tq_params_batch(src, n_workers, num_levels, mode, gamma, alpha_rule, alpha_user,
+                                 C.cast(out, C.c_void_p)), "tq_params_batch")
+    return out
 
 
 def tq_params_from_levels(levels: Sequence[float], mode: int = NONUNIFORM) -> Params:

@@ -169,3 +169,11 @@ extern "C" tq_status tq_params(const tq_stats_t* st, uint32_t num_levels, tq_mod
     out->levels[si] = alpha_f;
     return finish(out);
 }
+
+extern "C" tq_status tq_params_batch(const tq_stats_t* st, uint32_t n_workers, uint32_t num_levels, tq_mode mode,
+                                     double gamma, tq_alpha_rule rule, double alpha_user, tq_params_t* out) {
+    if (!st || !out || n_workers == 0 || n_workers > TQ_MAX_WORKERS) return TQ_ERR_INVALID_ARG;
+    for (uint32_t i = 0; i < n_workers; ++i)
+        if (tq_status s = tq_params(st + i, num_levels, mode, gamma, rule, alpha_user, out + i)) return s;
+    return TQ_OK;
+}

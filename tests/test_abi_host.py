@@ -122,6 +122,21 @@ def test_tq_params_errors(tq):
     assert e.value.status == tq.ERR_DOMAIN
 
 
+def test_params_batch_equals_single_calls(tq):
+    sts = [_stats(tq.Stats, g_min=1e-3 * (1 + i), n_tail=200_000 + 1000 * i) for i in range(5)]
+    arr = (tq.Stats * 5)(*sts)
+    out = tq.tq_params_batch(arr, 5, 16, tq.NONUNIFORM, 3.0)
+    for i in range(5):
+        one = tq.tq_params(sts[i], 16, tq.NONUNIFORM, 3.0)
+        assert bytes(out[i]) == bytes(one)
+    raw = b"".join(bytes(s) for s in sts)
+    again = tq.tq_params_batch(raw, 5, 16, tq.NONUNIFORM, 3.0)
+    assert bytes(again) == bytes(out)
+    with pytest.raises(tq.TqError) as e:
+        tq.tq_params_batch(arr, 5, 16, tq.NONUNIFORM, 1.5)
+    assert e.value.status == tq.ERR_DOMAIN
+
+
 def test_params_from_levels_agrees_with_oracle(tq, orc):
     lv = [-2.0, -0.5, -0.1, -0.01, 0.01, 0.1, 0.5, 2.0]
     a, b = tq.tq_params_from_levels(lv), orc.table_params(lv)
