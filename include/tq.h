@@ -57,7 +57,8 @@ typedef enum {
     TQ_ALPHA_USER = 2          /* caller supplies alpha */
 } tq_alpha_rule;
 
-enum { TQ_FLAG_ALPHA_CAPPED = 1, TQ_FLAG_ALPHA_AT_GMIN = 2, TQ_FLAG_GAMMA_FROM_MLE = 4 };
+enum { TQ_FLAG_ALPHA_CAPPED = 1, TQ_FLAG_ALPHA_AT_GMIN = 2, TQ_FLAG_GAMMA_FROM_MLE = 4,
+       TQ_FLAG_INVALID = 8 /* set by tq_params_device when a worker's statistics are outside the domain */ };
 
 /* Statistics of one worker's gradient; 64 bytes, written on the device by tq_stats. */
 typedef struct {
@@ -197,6 +198,34 @@ tq_status tq_compress(const void* grad_dev, tq_dtype dtype, uint64_t d, uint64_t
 tq_status tq_decompress_aggregate(const uint32_t* packed_dev, size_t words_stride, uint32_t n_workers,
                                   uint64_t d, const tq_params_t* params_host, const float* weights_host,
                                   float* out_dev, void* stream);
+
+/*
+ * The same round without a host round trip (the paper takes alpha and lambda_s as given inputs of
+ * Algorithm 1; where they come from -- Section 4 -- can equally run on the device).
+ *
+ * tq_params_device: Section 4 for n_workers records, one device thread per worker, same formulas and
+ *   arguments as tq_params, reading stats_dev and writing params_dev (both device memory, 8-byte
+ *   aligned).  Nothing is returned to the host: a worker whose statistics are outside the model's
+ *   domain gets flags = TQ_FLAG_INVALID, iterations = the tq_status it would have returned, alpha = 0
+ *   and an all-zero codebook; tq_compress_device_params then writes an all-zero row for it and the
+ *   aggregate receives zeros from it.  Device and host math libraries may differ in the last fp32 bit
+ *   of alpha or a level.
+ * tq_compress_device_params / tq_decompress_aggregate_device_params: as tq_compress /
+ *   tq_decompress_aggregate with params_dev[n_workers] in device memory; bits and mode are not read
+ *   from the records but given by the caller (num_levels, mode).
+ * All three only enqueue work on `stream`.  Errors: INVALID_ARG, DOMAIN (alpha_user <= 0), ALIGNMENT,
+ * BUFFER_TOO_SMALL, CUDA.
+ */
+tq_status tq_params_device(const tq_stats_t* stats_dev, uint32_t n_workers, uint32_t num_levels, tq_mode mode,
+                           double gamma, tq_alpha_rule alpha_rule, double alpha_user, tq_params_t* params_dev,
+                           void* stream);
+tq_status tq_compress_device_params(const void* grad_dev, tq_dtype dtype, uint64_t d, uint64_t grad_stride,
+                                    uint32_t n_workers, const tq_params_t* params_dev, uint32_t num_levels, tq_mode mode,
+                                    uint64_t seed, uint32_t first_worker, uint32_t* packed_dev, size_t words_stride,
+                                    void* stream);
+tq_status tq_decompress_aggregate_device_params(const uint32_t* packed_dev, size_t words_stride, uint32_t n_workers,
+                                                uint64_t d, const tq_params_t* params_dev, uint32_t num_levels,
+                                                const float* weights_host, float* out_dev, void* stream);
 
 const char* tq_strerror(tq_status status);
 int tq_last_cuda_error(void);   /* cudaError_t of the last failed runtime call on this thread, else 0 */

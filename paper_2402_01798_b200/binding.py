@@ -23,9 +23,10 @@ STATIC_MAX_WORKERS = 16
 F32, BF16 = 0, 1
 UNIFORM, NONUNIFORM = 0, 1
 ALPHA_CLOSED, ALPHA_FIXED_POINT, ALPHA_USER = 0, 1, 2
-FLAG_ALPHA_CAPPED, FLAG_ALPHA_AT_GMIN, FLAG_GAMMA_FROM_MLE = 1, 2, 4
+FLAG_ALPHA_CAPPED, FLAG_ALPHA_AT_GMIN, FLAG_GAMMA_FROM_MLE, FLAG_INVALID = 1, 2, 4, 8
 
-EXPORTS = ("tq_packed_words", "tq_stats_workspace_bytes", "tq_stats", "tq_stats_static", "tq_params", "tq_params_batch", "tq_params_from_levels",
+EXPORTS = ("tq_packed_words", "tq_stats_workspace_bytes", "tq_stats", "tq_stats_static", "tq_params", "tq_params_batch", "tq_params_from_levels", "tq_params_device",
+           "tq_compress_device_params", "tq_decompress_aggregate_device_params",
            "tq_compress", "tq_decompress_aggregate", "tq_strerror", "tq_last_cuda_error", "tq_kernel_launches")
 
 
@@ -80,6 +81,12 @@ def lib() -> C.CDLL:
         L.tq_compress.restype = C.c_int
         L.tq_decompress_aggregate.argtypes = [vp, sz, u32, u64, C.POINTER(Params), C.POINTER(f32), vp, vp]
         L.tq_decompress_aggregate.restype = C.c_int
+        L.tq_params_device.argtypes = [vp, u32, u32, C.c_int, f64, C.c_int, f64, vp, vp]
+        L.tq_params_device.restype = C.c_int
+        L.tq_compress_device_params.argtypes = [vp, C.c_int, u64, u64, u32, vp, u32, C.c_int, u64, u32, vp, sz, vp]
+        L.tq_compress_device_params.restype = C.c_int
+        L.tq_decompress_aggregate_device_params.argtypes = [vp, sz, u32, u64, vp, u32, C.POINTER(f32), vp, vp]
+        L.tq_decompress_aggregate_device_params.restype = C.c_int
         L.tq_strerror.argtypes = [C.c_int]; L.tq_strerror.restype = C.c_char_p
         L.tq_last_cuda_error.restype = C.c_int
         L.tq_kernel_launches.restype = u64
@@ -233,6 +240,52 @@ def tq_decompress_aggregate(packed: torch.Tensor, d: int, params: Sequence[Param
     words_stride = packed.stride(0) if n > 1 else packed.shape[1]
     _check(lib().tq_decompress_aggregate(packed.data_ptr(), words_stride, n, d, _params_array(params), w,
                                          out.data_ptr(), _stream(stream)), "tq_decompress_aggregate")
+    return out
+
+
+def tq_params_device(stats_dev: torch.Tensor, n_workers: int, num_levels: int, mode: int, gamma: float = math.nan,
+                     alpha_rule: int = ALPHA_FIXED_POINT, alpha_user: float = 0.0,
+                     params_dev: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Enqueue the parameter design on the device; returns the device tensor of n_workers 176-byte records."""
+    if params_dev is None:
+        params_dev = torch.empty(n_workers * C.sizeof(Params), dtype=torch.uint8, device=stats_dev.device)
+    _check(lib().tq_params_device(stats_dev.data_ptr(), n_workers, num_levels, mode, gamma, alpha_rule, alpha_user,
+                                  params_dev.data_ptr(), _stream(stream)), "tq_params_device")
+    return params_dev
+
+
+def params_to_host(params_dev: torch.Tensor):
+    """Copy device parameter records back (synchronises) and view them as Params structures."""
+    raw = params_dev.cpu().numpy().tobytes()
+    sz = C.sizeof(Params)
+    return [Params.from_buffer_copy(raw[i * sz:(i + 1) * sz]) for i in range(len(raw) // sz)]
+
+
+def tq_compress_device_params(grad: torch.Tensor, params_dev: torch.Tensor, num_levels: int, mode: int, seed: int,
+                              first_worker: int = 0, d: Optional[int] = None, packed: Optional[torch.Tensor] = None,
+                              stream=None) -> torch.Tensor:
+    n, d, stride = _grad_layout(grad, d)
+    bits = {2: 1, 4: 2, 8: 3, 16: 4}[num_levels]
+    if packed is None:
+        packed = torch.empty((n, tq_packed_words(d, bits)), dtype=torch.int32, device=grad.device)
+    words_stride = packed.stride(0) if packed.dim() == 2 and n > 1 else packed.shape[-1]
+    _check(lib().tq_compress_device_params(grad.data_ptr(), _dtype_code(grad), d, stride, n, params_dev.data_ptr(),
+                                           num_levels, mode, seed & 0xFFFFFFFFFFFFFFFF, first_worker, packed.data_ptr(),
+                                           words_stride, _stream(stream)), "tq_compress_device_params")
+    return packed
+
+
+def tq_decompress_aggregate_device_params(packed: torch.Tensor, d: int, params_dev: torch.Tensor, num_levels: int,
+                                          weights: Optional[Sequence[float]] = None,
+                                          out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    n = packed.shape[0]
+    if out is None:
+        out = torch.empty(d, dtype=torch.float32, device=packed.device)
+    w = None if weights is None else (C.c_float * n)(*[float(x) for x in weights])
+    words_stride = packed.stride(0) if n > 1 else packed.shape[1]
+    _check(lib().tq_decompress_aggregate_device_params(packed.data_ptr(), words_stride, n, d, params_dev.data_ptr(),
+                                                       num_levels, w, out.data_ptr(), _stream(stream)),
+           "tq_decompress_aggregate_device_params")
     return out
 
 

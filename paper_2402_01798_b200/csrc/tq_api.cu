@@ -99,7 +99,7 @@ tq_status tq_compress(const void* grad_dev, tq_dtype dtype, uint64_t d, uint64_t
     if (!aligned(packed_dev, 16) || words_stride % 4 != 0) return TQ_ERR_ALIGNMENT;
     if (words_stride < need) return TQ_ERR_BUFFER_TOO_SMALL;
     if (d == 0) return TQ_OK;
-    tq::CompressCall c{grad_dev, dtype == TQ_BF16, d, grad_stride, n_workers, params_host, bits,
+    tq::CompressCall c{grad_dev, dtype == TQ_BF16, d, grad_stride, n_workers, params_host, nullptr, bits,
                        params_host[0].mode == TQ_NONUNIFORM, seed, first_worker, packed_dev, words_stride, need,
                        static_cast<cudaStream_t>(stream)};
     const cudaError_t e = tq::launch_compress(c);
@@ -119,7 +119,62 @@ tq_status tq_decompress_aggregate(const uint32_t* packed_dev, size_t words_strid
     if (!aligned(packed_dev, 16) || words_stride % 4 != 0 || !aligned(out_dev, 32)) return TQ_ERR_ALIGNMENT;
     if (words_stride < need) return TQ_ERR_BUFFER_TOO_SMALL;
     if (d == 0) return TQ_OK;
-    tq::DecompressCall c{packed_dev, words_stride, need, n_workers, d, params_host, weights_host, bits, out_dev,
+    tq::DecompressCall c{packed_dev, words_stride, need, n_workers, d, params_host, nullptr, weights_host, bits, out_dev,
+                         static_cast<cudaStream_t>(stream)};
+    const cudaError_t e = tq::launch_decompress(c);
+    if (e != cudaSuccess) return cuda_failed(e);
+    g_launches += 1;
+    return TQ_OK;
+}
+
+tq_status tq_params_device(const tq_stats_t* stats_dev, uint32_t n_workers, uint32_t num_levels, tq_mode mode,
+                           double gamma, tq_alpha_rule alpha_rule, double alpha_user, tq_params_t* params_dev,
+                           void* stream) {
+    uint32_t bits = 0;
+    if (!stats_dev || !params_dev || n_workers == 0 || n_workers > TQ_MAX_WORKERS) return TQ_ERR_INVALID_ARG;
+    if (!tq::params_request_ok(num_levels, mode, alpha_rule, &bits)) return TQ_ERR_INVALID_ARG;
+    if (alpha_rule == TQ_ALPHA_USER && !(alpha_user > 0.0)) return TQ_ERR_DOMAIN;
+    if (!aligned(stats_dev, 8) || !aligned(params_dev, 8)) return TQ_ERR_ALIGNMENT;
+    const cudaError_t e = tq::launch_params_device(stats_dev, n_workers, num_levels, bits, mode, gamma, alpha_rule,
+                                                   alpha_user, params_dev, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_failed(e);
+    g_launches += 1;
+    return TQ_OK;
+}
+
+tq_status tq_compress_device_params(const void* grad_dev, tq_dtype dtype, uint64_t d, uint64_t grad_stride,
+                                    uint32_t n_workers, const tq_params_t* params_dev, uint32_t num_levels, tq_mode mode,
+                                    uint64_t seed, uint32_t first_worker, uint32_t* packed_dev, size_t words_stride,
+                                    void* stream) {
+    if (tq_status s = check_grad(grad_dev, dtype, d, grad_stride, n_workers)) return s;
+    uint32_t bits = 0;
+    if (!params_dev || !tq::params_request_ok(num_levels, mode, TQ_ALPHA_CLOSED, &bits)) return TQ_ERR_INVALID_ARG;
+    const size_t need = tq_packed_words(d, bits);
+    if (need && !packed_dev) return TQ_ERR_INVALID_ARG;
+    if (!aligned(packed_dev, 16) || words_stride % 4 != 0 || !aligned(params_dev, 8)) return TQ_ERR_ALIGNMENT;
+    if (words_stride < need) return TQ_ERR_BUFFER_TOO_SMALL;
+    if (d == 0) return TQ_OK;
+    tq::CompressCall c{grad_dev, dtype == TQ_BF16, d, grad_stride, n_workers, nullptr, params_dev, bits,
+                       mode == TQ_NONUNIFORM, seed, first_worker, packed_dev, words_stride, need,
+                       static_cast<cudaStream_t>(stream)};
+    const cudaError_t e = tq::launch_compress(c);
+    if (e != cudaSuccess) return cuda_failed(e);
+    g_launches += 1;
+    return TQ_OK;
+}
+
+tq_status tq_decompress_aggregate_device_params(const uint32_t* packed_dev, size_t words_stride, uint32_t n_workers,
+                                                uint64_t d, const tq_params_t* params_dev, uint32_t num_levels,
+                                                const float* weights_host, float* out_dev, void* stream) {
+    if (n_workers == 0 || n_workers > TQ_MAX_WORKERS || d > (1ull << 40)) return TQ_ERR_INVALID_ARG;
+    uint32_t bits = 0;
+    if (!params_dev || !tq::params_request_ok(num_levels, TQ_UNIFORM, TQ_ALPHA_CLOSED, &bits)) return TQ_ERR_INVALID_ARG;
+    const size_t need = tq_packed_words(d, bits);
+    if (d && (!packed_dev || !out_dev)) return TQ_ERR_INVALID_ARG;
+    if (!aligned(packed_dev, 16) || words_stride % 4 != 0 || !aligned(out_dev, 32) || !aligned(params_dev, 8)) return TQ_ERR_ALIGNMENT;
+    if (words_stride < need) return TQ_ERR_BUFFER_TOO_SMALL;
+    if (d == 0) return TQ_OK;
+    tq::DecompressCall c{packed_dev, words_stride, need, n_workers, d, nullptr, params_dev, weights_host, bits, out_dev,
                          static_cast<cudaStream_t>(stream)};
     const cudaError_t e = tq::launch_decompress(c);
     if (e != cudaSuccess) return cuda_failed(e);

@@ -42,6 +42,8 @@ struct CompressArgs {
 
 enum Search { kUniform = 0, kGrid = 1, kBinary = 2 };
 
+cudaError_t launch_compress_dev(const CompressCall& c);
+
 __device__ __forceinline__ float mul_sat(float a, float b) {
     float r; asm("mul.rn.sat.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b)); return r;
 }
@@ -264,18 +266,14 @@ __device__ __forceinline__ void compress_run(const char* row, uint32_t* prow, ui
 #define TQ_COMPRESS_MIN_BLOCKS 4
 #endif
 
+// Per-block set-up of the shared tables for quantizer q, then the block's share of worker wi's runs.
+// s_grid must hold kMaxGridCells + 1 entries when SEARCH == kGrid.
 template <int BITS, int SEARCH, bool BF16>
-__global__ void __launch_bounds__(kThreads, TQ_COMPRESS_MIN_BLOCKS)
-compress_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
-                const __grid_constant__ CompressArgs args, const __grid_constant__ RoundKeys rk,
-                uint32_t first_worker, uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_out) {
+__device__ __forceinline__ void compress_block(const WorkerQ& q, float2* s_grid, float2* s_cell, float* s_search,
+                                               const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
+                                               const RoundKeys& rk, uint32_t worker, uint32_t wi,
+                                               uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_out) {
     constexpr int L = 1 << BITS;
-    const uint32_t wi = blockIdx.y;
-    const WorkerQ& q = args.q[wi];
-
-    __shared__ __align__(16) float2 s_grid[SEARCH == kGrid ? kMaxGridCells + 1 : 1];
-    __shared__ __align__(16) float2 s_cell[TQ_MAX_LEVELS];
-    __shared__ float s_search[2 * TQ_MAX_LEVELS];
     if constexpr (SEARCH != kUniform) {
         if (threadIdx.x < L - 1) s_cell[threadIdx.x] = make_float2(q.levels[threadIdx.x], q.inv_width[threadIdx.x]);
     }
@@ -284,7 +282,7 @@ compress_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
             s_search[threadIdx.x] = (threadIdx.x >= 1 && threadIdx.x <= L - 2) ? q.levels[threadIdx.x] : __int_as_float(0x7F800000);
     }
     if constexpr (SEARCH == kGrid) {
-        // cells of the interior levels l_1 .. l_{s-1} (distinct by the host's choice of M)
+        // cells of the interior levels l_1 .. l_{s-1} (distinct by the choice of M)
         uint32_t lc[L];
 #pragma unroll
         for (int j = 1; j <= L - 2; ++j)
@@ -304,19 +302,106 @@ compress_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
     constexpr size_t esz = BF16 ? 2 : 4;
     const char* row = static_cast<const char*>(grad) + static_cast<uint64_t>(wi) * grad_stride * esz;
     uint32_t* prow = packed + static_cast<uint64_t>(wi) * words_stride;
-    const uint32_t worker = first_worker + wi;
     const uint64_t n_runs = (d + 31) >> 5;
-    const uint64_t full_runs = d >> 5;
     const RunCtx cx{q.alpha, q.inv_step, q.top, q.inv_2alpha, q.cell_scale, reinterpret_cast<const char*>(s_grid),
                     reinterpret_cast<const char*>(s_cell), s_search};
     const uint64_t stride = static_cast<uint64_t>(gridDim.x) * kThreads;
 
     uint64_t run = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x;
-    const uint64_t interior = full_runs == n_runs ? n_runs - 1 : full_runs;    // runs that are full AND not the row's last
+    const uint64_t interior = n_runs - 1;      // every run before the row's last one is full
     for (; run < interior; run += stride)
         compress_run<BITS, SEARCH, BF16, false>(row, prow, run, d, words_out, worker, rk, cx);
     if (run == n_runs - 1)
         compress_run<BITS, SEARCH, BF16, true>(row, prow, run, d, words_out, worker, rk, cx);
+}
+
+// Quantizers passed by value in the kernel's parameter space (host-side tq_params).
+template <int BITS, int SEARCH, bool BF16>
+__global__ void __launch_bounds__(kThreads, TQ_COMPRESS_MIN_BLOCKS)
+compress_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
+                const __grid_constant__ CompressArgs args, const __grid_constant__ RoundKeys rk,
+                uint32_t first_worker, uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_out) {
+    __shared__ __align__(16) float2 s_grid[SEARCH == kGrid ? kMaxGridCells + 1 : 1];
+    __shared__ __align__(16) float2 s_cell[TQ_MAX_LEVELS];
+    __shared__ float s_search[2 * TQ_MAX_LEVELS];
+    const uint32_t wi = blockIdx.y;
+    compress_block<BITS, SEARCH, BF16>(args.q[wi], s_grid, s_cell, s_search, grad, d, grad_stride, rk, first_worker + wi, wi,
+                                       packed, words_stride, words_out);
+}
+
+// Out-of-line copy of the binary-search block for the run-time fallback of compress_kernel_dev, so
+// that the rarely taken path does not compete for registers with the grid path.
+template <int BITS, bool BF16>
+__device__ __noinline__ void compress_block_binary(const WorkerQ& q, float2* s_grid, float2* s_cell, float* s_search,
+                                                   const void* grad, uint64_t d, uint64_t grad_stride, const RoundKeys& rk,
+                                                   uint32_t worker, uint32_t wi, uint32_t* packed, uint64_t words_stride,
+                                                   uint64_t words_out) {
+    compress_block<BITS, kBinary, BF16>(q, s_grid, s_cell, s_search, grad, d, grad_stride, rk, worker, wi, packed,
+                                        words_stride, words_out);
+}
+
+// The grid cell of a value as a plain integer (device copy of the host's cell_of).
+__device__ __forceinline__ uint32_t cell_index(float g, float alpha, float inv_2alpha, uint32_t cells) {
+    return __float_as_uint(grid_cell(g, alpha, inv_2alpha, ldexpf(static_cast<float>(cells), -149)));
+}
+
+// Quantizers read from device memory (tq_params_device): no host round trip before the launch.
+// Thread 0 turns worker wi's tq_params_t into the kernel's WorkerQ, including the choice of the lookup
+// grid; a worker marked invalid (alpha = 0) gets an all-zero row.  NONUNIFORM: the grid search, or the
+// binary search when no grid separates the levels, chosen per block at run time.
+template <int BITS, bool NONUNIFORM, bool BF16>
+__global__ void __launch_bounds__(kThreads, TQ_COMPRESS_MIN_BLOCKS)
+compress_kernel_dev(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
+                    const tq_params_t* __restrict__ params, const __grid_constant__ RoundKeys rk,
+                    uint32_t first_worker, uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_out) {
+    __shared__ __align__(16) float2 s_grid[NONUNIFORM ? kMaxGridCells + 1 : 1];
+    __shared__ __align__(16) float2 s_cell[TQ_MAX_LEVELS];
+    __shared__ float s_search[2 * TQ_MAX_LEVELS];
+    __shared__ WorkerQ s_q;
+    const uint32_t wi = blockIdx.y;
+    if (threadIdx.x < TQ_MAX_LEVELS) {
+        s_q.levels[threadIdx.x] = params[wi].levels[threadIdx.x];
+        s_q.inv_width[threadIdx.x] = params[wi].inv_width[threadIdx.x];
+    }
+    if (threadIdx.x == 0) {
+        const tq_params_t& p = params[wi];
+        const bool ok = p.alpha > 0.0f && p.bits == BITS && !(p.flags & TQ_FLAG_INVALID);
+        s_q.alpha = ok ? p.alpha : 0.0f;
+        s_q.inv_step = p.inv_step;
+        s_q.top = static_cast<float>((1 << BITS) - 1);
+        s_q.inv_2alpha = ok ? __fdiv_rn(1.0f, __fmul_rn(2.0f, p.alpha)) : 0.0f;
+        uint32_t cells = 0;
+        if (NONUNIFORM && ok && s_q.inv_2alpha <= 3.402823466e38f) {
+            constexpr int s = (1 << BITS) - 1;
+            for (uint32_t m = kMinGridCells; m <= static_cast<uint32_t>(kMaxGridCells) && cells == 0; m *= 2) {
+                bool distinct = true;
+                for (int j = 2; j <= s - 1 && distinct; ++j)
+                    distinct = cell_index(p.levels[j], p.alpha, s_q.inv_2alpha, m) > cell_index(p.levels[j - 1], p.alpha, s_q.inv_2alpha, m);
+                if (distinct) cells = m;
+            }
+        }
+        s_q.cells = cells;
+        s_q.cell_scale = ldexpf(static_cast<float>(cells), -149);
+    }
+    __syncthreads();
+    if (!(s_q.alpha > 0.0f)) {       // invalid parameters: the row is all code 0
+        uint32_t* prow = packed + static_cast<uint64_t>(wi) * words_stride;
+        for (uint64_t w = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x; w < words_out;
+             w += static_cast<uint64_t>(gridDim.x) * kThreads)
+            prow[w] = 0u;
+        return;
+    }
+    if constexpr (!NONUNIFORM) {
+        compress_block<BITS, kUniform, BF16>(s_q, s_grid, s_cell, s_search, grad, d, grad_stride, rk, first_worker + wi, wi,
+                                             packed, words_stride, words_out);
+    } else {
+        if (s_q.cells != 0)
+            compress_block<BITS, kGrid, BF16>(s_q, s_grid, s_cell, s_search, grad, d, grad_stride, rk, first_worker + wi, wi,
+                                              packed, words_stride, words_out);
+        else
+            compress_block_binary<BITS, BF16>(s_q, s_grid, s_cell, s_search, grad, d, grad_stride, rk, first_worker + wi, wi,
+                                              packed, words_stride, words_out);
+    }
 }
 
 // ---- host side ---------------------------------------------------------------------------------------
@@ -341,13 +426,32 @@ static uint32_t choose_cells(const tq_params_t& p, float inv_2alpha) {
     return 0;
 }
 
+static RoundKeys round_keys(uint64_t seed) {
+    RoundKeys rk;
+    uint32_t k0 = static_cast<uint32_t>(seed), k1 = static_cast<uint32_t>(seed >> 32);
+    for (int r = 0; r < 10; ++r) { rk.k0[r] = k0; rk.k1[r] = k1; k0 += 0x9E3779B9u; k1 += 0xBB67AE85u; }
+    return rk;
+}
+
+// Persistent grid: 4 resident blocks per SM spread over the workers (table modes build their lookup
+// grid once per block); uniform mode has no per-block set-up, so one block per tile lets the hardware
+// scheduler balance the tail.
+static dim3 compress_grid(uint64_t d, uint32_t n_workers, bool persistent) {
+    const uint64_t n_runs = (d + 31) >> 5;
+    const uint64_t tiles = (n_runs + kThreads - 1) / kThreads;
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    uint64_t per_worker = (static_cast<uint64_t>(sms) * TQ_COMPRESS_MIN_BLOCKS + n_workers - 1) / n_workers;
+    if (!persistent || per_worker > tiles) per_worker = tiles;
+    if (per_worker > 0x7FFFFFFFull) per_worker = 0x7FFFFFFFull;
+    if (per_worker < 1) per_worker = 1;
+    return dim3(static_cast<unsigned>(per_worker), n_workers);
+}
+
 template <int BITS, int SEARCH, bool BF>
 static cudaError_t launch(const CompressCall& c, const CompressArgs& args, dim3 grid) {
-    RoundKeys rk;
-    uint32_t k0 = static_cast<uint32_t>(c.seed), k1 = static_cast<uint32_t>(c.seed >> 32);
-    for (int r = 0; r < 10; ++r) { rk.k0[r] = k0; rk.k1[r] = k1; k0 += 0x9E3779B9u; k1 += 0xBB67AE85u; }
     compress_kernel<BITS, SEARCH, BF><<<grid, kThreads, 0, c.stream>>>(
-        c.grad, c.d, c.grad_stride, args, rk, c.first_worker, c.packed, c.words_stride, c.words_out);
+        c.grad, c.d, c.grad_stride, args, round_keys(c.seed), c.first_worker, c.packed, c.words_stride, c.words_out);
     return cudaGetLastError();
 }
 
@@ -359,6 +463,8 @@ static cudaError_t dispatch(const CompressCall& c, const CompressArgs& a, dim3 g
 }
 
 cudaError_t launch_compress(const CompressCall& c) {
+    if (c.d == 0) return cudaSuccess;
+    if (c.params_dev) return launch_compress_dev(c);
     static thread_local CompressArgs args;   // 9 KB: keep it off the stack
     int search = c.nonuniform ? kGrid : kUniform;
     for (uint32_t i = 0; i < c.n_workers; ++i) {
@@ -374,24 +480,34 @@ cudaError_t launch_compress(const CompressCall& c) {
             if (q.cells == 0 || !std::isfinite(q.inv_2alpha)) search = kBinary;
         }
     }
-    const uint64_t n_runs = (c.d + 31) >> 5;
-    const uint64_t tiles = (n_runs + kThreads - 1) / kThreads;
-    if (tiles == 0) return cudaSuccess;
-    // Table modes: persistent blocks (the lookup grid is built once per block), 4 resident blocks per
-    // SM over all workers.  Uniform mode has no per-block set-up, so one block per tile lets the
-    // hardware scheduler balance the tail.
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    uint64_t per_worker = (static_cast<uint64_t>(sms) * TQ_COMPRESS_MIN_BLOCKS + c.n_workers - 1) / c.n_workers;
-    if (search == kUniform || per_worker > tiles) per_worker = tiles;
-    if (per_worker > 0x7FFFFFFFull) per_worker = 0x7FFFFFFFull;
-    if (per_worker < 1) per_worker = 1;
-    const dim3 grid(static_cast<unsigned>(per_worker), c.n_workers);
+    const dim3 grid = compress_grid(c.d, c.n_workers, search != kUniform);
     switch (c.bits) {
         case 1: return dispatch<1>(c, args, grid, search);
         case 2: return dispatch<2>(c, args, grid, search);
         case 3: return dispatch<3>(c, args, grid, search);
         default: return dispatch<4>(c, args, grid, search);
+    }
+}
+
+template <int BITS, bool NU, bool BF>
+static cudaError_t launch_dev(const CompressCall& c, dim3 grid) {
+    compress_kernel_dev<BITS, NU, BF><<<grid, kThreads, 0, c.stream>>>(
+        c.grad, c.d, c.grad_stride, c.params_dev, round_keys(c.seed), c.first_worker, c.packed, c.words_stride, c.words_out);
+    return cudaGetLastError();
+}
+template <int BITS>
+static cudaError_t dispatch_dev(const CompressCall& c, dim3 grid) {
+    if (c.nonuniform) return c.bf16 ? launch_dev<BITS, true, true>(c, grid) : launch_dev<BITS, true, false>(c, grid);
+    return c.bf16 ? launch_dev<BITS, false, true>(c, grid) : launch_dev<BITS, false, false>(c, grid);
+}
+
+cudaError_t launch_compress_dev(const CompressCall& c) {
+    const dim3 grid = compress_grid(c.d, c.n_workers, c.nonuniform);
+    switch (c.bits) {
+        case 1: return dispatch_dev<1>(c, grid);
+        case 2: return dispatch_dev<2>(c, grid);
+        case 3: return dispatch_dev<3>(c, grid);
+        default: return dispatch_dev<4>(c, grid);
     }
 }
 

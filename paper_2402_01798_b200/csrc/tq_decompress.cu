@@ -17,6 +17,12 @@ namespace tq {
 struct DecompressArgs {
     float table[TQ_MAX_WORKERS][TQ_MAX_LEVELS];   // levels, already multiplied by w_i when weights are given
 };
+// Device-resident parameters: the codebooks are read from params_dev by each block; weights by value.
+struct DeviceTables {
+    const tq_params_t* params_dev;    // nullptr: use DecompressArgs
+    int use_weights;
+    float weights[TQ_MAX_WORKERS];
+};
 
 __device__ __forceinline__ uint32_t ldg32_stream(const uint32_t* p) {
     uint32_t v;
@@ -116,7 +122,8 @@ __device__ __forceinline__ void add_unit(f32x2* acc, uint32_t f, const char* tab
 template <int BITS>
 __global__ void __launch_bounds__(kThreads, TQ_DECOMPRESS_MIN_BLOCKS)
 decompress_kernel(const uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_valid, uint32_t n,
-                  uint64_t d, const __grid_constant__ DecompressArgs args, float scale, int divide,
+                  uint64_t d, const __grid_constant__ DecompressArgs args, const __grid_constant__ DeviceTables dt,
+                  float scale, int divide,
                   float* __restrict__ out) {
     constexpr int E = Unit<BITS>::kElems, U = Unit<BITS>::kUnits;
 
@@ -124,8 +131,17 @@ decompress_kernel(const uint32_t* __restrict__ packed, uint64_t words_stride, ui
     // (code * 4 < 64) can be merged into the worker's base offset by the same byte-permute that
     // extracts it.  Bank = code: the lookups of one instruction never conflict.
     __shared__ __align__(256) float s_tab[TQ_MAX_WORKERS * kTabStride];
-    for (uint32_t t = threadIdx.x; t < n * TQ_MAX_LEVELS; t += kThreads)
-        s_tab[(t / TQ_MAX_LEVELS) * kTabStride + t % TQ_MAX_LEVELS] = args.table[t / TQ_MAX_LEVELS][t % TQ_MAX_LEVELS];
+    for (uint32_t t = threadIdx.x; t < n * TQ_MAX_LEVELS; t += kThreads) {
+        const uint32_t i = t / TQ_MAX_LEVELS, k = t % TQ_MAX_LEVELS;
+        float v;
+        if (dt.params_dev) {     // same rounded product w_i * l as the host forms for the by-value table
+            const float l = dt.params_dev[i].levels[k];
+            v = dt.use_weights ? __fmul_rn(dt.weights[i], l) : l;
+        } else {
+            v = args.table[i][k];
+        }
+        s_tab[i * kTabStride + k] = v;
+    }
     __syncthreads();
     const char* tab_bytes = reinterpret_cast<const char*>(s_tab);
 
@@ -198,26 +214,32 @@ decompress_kernel(const uint32_t* __restrict__ packed, uint64_t words_stride, ui
 }
 
 template <int BITS>
-static cudaError_t launch(const DecompressCall& c, const DecompressArgs& args, float scale, int divide) {
+static cudaError_t launch(const DecompressCall& c, const DecompressArgs& args, const DeviceTables& dt, float scale, int divide) {
     const uint64_t n_units = (c.d + Unit<BITS>::kElems - 1) / Unit<BITS>::kElems;
     const uint64_t per_block = static_cast<uint64_t>(kThreads) * Unit<BITS>::kUnits;
     const uint64_t blocks = (n_units + per_block - 1) / per_block;
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7FFFFFFFull) return cudaErrorInvalidConfiguration;
     decompress_kernel<BITS><<<static_cast<unsigned>(blocks), kThreads, 0, c.stream>>>(
-        c.packed, c.words_stride, c.words_valid, c.n_workers, c.d, args, scale, divide, c.out);
+        c.packed, c.words_stride, c.words_valid, c.n_workers, c.d, args, dt, scale, divide, c.out);
     return cudaGetLastError();
 }
 
 cudaError_t launch_decompress(const DecompressCall& c) {
     static thread_local DecompressArgs args;
-    for (uint32_t i = 0; i < c.n_workers; ++i)
+    static thread_local DeviceTables dt;
+    dt.params_dev = c.params_dev;
+    dt.use_weights = c.weights ? 1 : 0;
+    for (uint32_t i = 0; i < c.n_workers; ++i) {
+        dt.weights[i] = c.weights ? c.weights[i] : 0.0f;
+        if (c.params_dev) continue;
         for (int k = 0; k < TQ_MAX_LEVELS; ++k) {
             const float l = c.params[i].levels[k];
             // weighted form: each product w_i * l is rounded to fp32 once; it depends on (i, k) only,
             // so it is formed here instead of once per element
             args.table[i][k] = c.weights ? c.weights[i] * l : l;
         }
+    }
     float scale = 1.0f;
     int divide = 0;
     if (!c.weights) {
@@ -226,10 +248,10 @@ cudaError_t launch_decompress(const DecompressCall& c) {
         else { divide = 1; scale = static_cast<float>(n); }
     }
     switch (c.bits) {
-        case 1: return launch<1>(c, args, scale, divide);
-        case 2: return launch<2>(c, args, scale, divide);
-        case 3: return launch<3>(c, args, scale, divide);
-        default: return launch<4>(c, args, scale, divide);
+        case 1: return launch<1>(c, args, dt, scale, divide);
+        case 2: return launch<2>(c, args, dt, scale, divide);
+        case 3: return launch<3>(c, args, dt, scale, divide);
+        default: return launch<4>(c, args, dt, scale, divide);
     }
 }
 

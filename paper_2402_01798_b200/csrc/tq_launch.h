@@ -9,7 +9,9 @@ namespace tq {
 
 struct CompressCall {
     const void* grad; bool bf16; uint64_t d, grad_stride; uint32_t n_workers;
-    const tq_params_t* params; uint32_t bits; bool nonuniform;
+    const tq_params_t* params;       // host array, or
+    const tq_params_t* params_dev;   // device array (then bits / nonuniform come from the caller)
+    uint32_t bits; bool nonuniform;
     uint64_t seed; uint32_t first_worker;
     uint32_t* packed; uint64_t words_stride, words_out;
     cudaStream_t stream;
@@ -18,7 +20,9 @@ cudaError_t launch_compress(const CompressCall& c);
 
 struct DecompressCall {
     const uint32_t* packed; uint64_t words_stride, words_valid; uint32_t n_workers; uint64_t d;
-    const tq_params_t* params; const float* weights; uint32_t bits;
+    const tq_params_t* params;       // host array, or
+    const tq_params_t* params_dev;   // device array (then bits comes from the caller)
+    const float* weights; uint32_t bits;
     float* out; cudaStream_t stream;
 };
 cudaError_t launch_decompress(const DecompressCall& c);
@@ -33,5 +37,10 @@ size_t stats_workspace_bytes(uint32_t n_workers);
 // Same reduction with the library's built-in scratch array as workspace (c.workspace is ignored).
 // *limit is set when n_workers exceeds what the array holds; nothing is launched then.
 cudaError_t launch_stats_static(const StatsCall& c, int* launches, bool* limit);
+
+// Parameter design on the device (one thread per worker); request already validated by params_request_ok.
+bool params_request_ok(uint32_t num_levels, int mode, int rule, uint32_t* bits);
+cudaError_t launch_params_device(const tq_stats_t* stats_dev, uint32_t n, uint32_t num_levels, uint32_t bits, uint32_t mode,
+                                 double gamma, int rule, double alpha_user, tq_params_t* params_dev, cudaStream_t stream);
 
 }  // namespace tq

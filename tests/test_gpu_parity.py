@@ -355,3 +355,72 @@ def test_config5_billion_elements_windows(tq, orc):
     assert st[1].n_tail == o.n_tail and st[1].max_abs == o.max_abs
     assert math.isclose(st[1].sum_abs, o.sum_abs, rel_tol=TOL_SUM) and math.isclose(st[1].sum_sq, o.sum_sq, rel_tol=TOL_SUM)
     assert math.isclose(st[1].sum_log_tail, o.sum_log_tail, rel_tol=TOL_LOG)
+
+
+# ----------------------------------------------------------------------- device-resident parameters
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("L,mode,gamma", [(4, 0, 3.0), (8, 0, 2.5), (8, 1, 2.5), (16, 1, 3.0), (16, 1, 2.2), (2, 1, 4.0), (16, 0, float("nan"))])
+def test_round_without_host_round_trip(tq, orc, dtype, L, mode, gamma):
+    """statistics -> tq_params_device -> tq_compress_device_params -> tq_decompress_aggregate_device_params,
+    nothing copied to the host in between.  The device-made parameters agree with the host's (and so
+    with the oracle's) to fp32 rounding; codes and aggregate are bit-exact against the oracle run on
+    the device-made parameters."""
+    d, n = 300_007, 5
+    g = heavy_tailed(d, n, dtype, seed=L * 7 + mode)
+    stats_dev = tq.tq_stats(g, d)
+    params_dev = tq.tq_params_device(stats_dev, n, L, mode, gamma)
+    packed = tq.tq_compress_device_params(g, params_dev, L, mode, seed=321, first_worker=3, d=d)
+    out = tq.tq_decompress_aggregate_device_params(packed, d, params_dev, L)
+    torch.cuda.synchronize()
+    st = tq.stats_to_host(stats_dev)
+    dev_ps = tq.params_to_host(params_dev)
+    for s, p in zip(st, dev_ps):
+        h = tq.tq_params(s, L, mode, gamma)
+        assert p.flags == h.flags and p.bits == h.bits and p.mode == h.mode and p.iterations == h.iterations
+        assert math.isclose(p.alpha, h.alpha, rel_tol=3e-7) and math.isclose(p.inv_step, h.inv_step, rel_tol=5e-7)
+        assert np.allclose(list(p.levels), list(h.levels), rtol=5e-7, atol=0)
+        assert np.allclose(list(p.inv_width), list(h.inv_width), rtol=2e-6, atol=0)
+    ops = [to_oracle_params(orc, p) for p in dev_ps]
+    got = packed.cpu().numpy().view(np.uint32)
+    for i in range(n):
+        assert np.array_equal(got[i], orc.compress(host_f32(orc, g[i, :d]), ops[i], 321, 3 + i)), i
+    assert np.array_equal(out.cpu().numpy(), orc.decompress_aggregate(got, d, ops))
+    # the host-parameter path on the same (device-made) parameters gives the same bytes
+    again = tq.tq_compress(g, dev_ps, 321, 3, d=d)
+    assert torch.equal(again, packed)
+    w = [0.1 * (i + 1) for i in range(n)]
+    ow = tq.tq_decompress_aggregate_device_params(packed, d, params_dev, L, weights=w)
+    assert torch.equal(ow, tq.tq_decompress_aggregate(packed, d, dev_ps, weights=w))
+
+
+def test_device_params_marks_bad_statistics_and_fallback_codebooks(tq, orc):
+    """A worker whose statistics are outside the domain is flagged, its row is all zeros and it adds zero
+    to the aggregate; a crowded caller-made codebook written into the device records takes the
+    binary-search path inside the device-parameter kernel."""
+    d, n = 50_003, 3
+    g = heavy_tailed(d, n, torch.float32, seed=77)
+    g[1].zero_()                                             # all-zero gradient: g_min = 0, no tail
+    stats_dev = tq.tq_stats(g, d)
+    params_dev = tq.tq_params_device(stats_dev, n, 8, tq.NONUNIFORM, 3.0)
+    ps = tq.params_to_host(params_dev)
+    assert ps[1].flags & tq.FLAG_INVALID and ps[1].iterations == tq.ERR_DOMAIN and ps[1].alpha == 0.0
+    assert not (ps[0].flags & tq.FLAG_INVALID) and not (ps[2].flags & tq.FLAG_INVALID)
+    packed = tq.tq_compress_device_params(g, params_dev, 8, tq.NONUNIFORM, seed=5, d=d)
+    out = tq.tq_decompress_aggregate_device_params(packed, d, params_dev, 8)
+    got = packed.cpu().numpy().view(np.uint32)
+    assert not got[1].any()
+    ops = [to_oracle_params(orc, p) for p in ps]
+    for i in (0, 2):
+        assert np.array_equal(got[i], orc.compress(host_f32(orc, g[i, :d]), ops[i], 5, i))
+    acc = np.zeros(d, dtype=F32)
+    for i in range(n):
+        acc = (acc + np.array(ops[i].levels[:8], dtype=F32)[orc.unpack(got[i], d, 3)]).astype(F32)
+    assert np.array_equal(out.cpu().numpy(), (acc / F32(3)).astype(F32))
+    # crowded codebook -> binary-search fallback
+    lv = np.concatenate([[-1.0], np.linspace(0.3, 0.3001, 6), [1.0]]).astype(F32)
+    p = tq.tq_params_from_levels([float(x) for x in lv])
+    raw = torch.frombuffer(bytearray(bytes(p) * n), dtype=torch.uint8).cuda()
+    g2 = heavy_tailed(d, n, torch.float32, seed=78, scale=0.2)
+    pk = tq.tq_compress_device_params(g2, raw, 8, tq.NONUNIFORM, seed=9, d=d).cpu().numpy().view(np.uint32)
+    for i in range(n):
+        assert np.array_equal(pk[i], orc.compress(host_f32(orc, g2[i, :d]), to_oracle_params(orc, p), 9, i))
