@@ -2,9 +2,10 @@
 """Benchmark of the truncated-quantization hot path on B200.
 
 A step is one full round over one batch of synthetic heavy-tailed gradients already resident in
-HBM: statistics (two passes: moments, then the tail beyond g_min = mean|g|) -> record copied to the
-host -> closed-form parameters -> fused truncate + stochastic round + pack for all N workers ->
-fused unpack + dequantize + average.  Throughput is bytes of gradient input (N * d * elemsize) per
+HBM: statistics (two passes: moments, then the tail beyond g_min = mean|g|) -> closed-form
+parameters (on the device by default; --host-params copies the records back and designs them on the
+host) -> fused truncate + stochastic round + pack for all N workers -> fused unpack + dequantize +
+average.  Throughput is bytes of gradient input (N * d * elemsize) per
 second of step time.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config 0..4] [--impl ours|reference]
@@ -184,6 +185,8 @@ def main():
     ap.add_argument("--variant", type=int, default=None,
                     help="with --config 3: index 0..11 into the bf16 sweep (gamma x mode x levels)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--host-params", action="store_true",
+                    help="design the parameters on the host (statistics copied back, one sync per round)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -225,19 +228,31 @@ def main():
     ws = torch.empty(tq.tq_stats_workspace_bytes(N), dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
 
+    params_dev = torch.empty(N * 176, dtype=torch.uint8, device=dev)
+
     def one_round(ev=None):
+        """Returns what tq_decompress_aggregate needs to run again on this round's packed rows."""
         if ev: ev[0].record()
         tq.tq_stats(g, d, stats_dev=stats_dev, workspace=ws)
         if ev: ev[1].record()
-        stats_pin.copy_(stats_dev, non_blocking=True)
-        stream.synchronize()                                   # the only host sync of a round
-        ps = tq.tq_params_batch(stats_pin, N, w.num_levels, mode, w.gamma)
+        if args.host_params:
+            stats_pin.copy_(stats_dev, non_blocking=True)
+            stream.synchronize()                               # the one host sync of this variant of the round
+            ps = tq.tq_params_batch(stats_pin, N, w.num_levels, mode, w.gamma)
+            if ev: ev[2].record()
+            tq.tq_compress(g, ps, seed=1234, d=d, packed=packed)
+            if ev: ev[3].record()
+            tq.tq_decompress_aggregate(packed, d, ps, out=out)
+            if ev: ev[4].record()
+            return lambda: tq.tq_decompress_aggregate(packed, d, ps, out=out)
+        # default: parameters designed on the device, nothing returns to the host inside the round
+        tq.tq_params_device(stats_dev, N, w.num_levels, mode, w.gamma, params_dev=params_dev)
         if ev: ev[2].record()
-        tq.tq_compress(g, ps, seed=1234, d=d, packed=packed)
+        tq.tq_compress_device_params(g, params_dev, w.num_levels, mode, seed=1234, d=d, packed=packed)
         if ev: ev[3].record()
-        tq.tq_decompress_aggregate(packed, d, ps, out=out)
+        tq.tq_decompress_aggregate_device_params(packed, d, params_dev, w.num_levels, out=out)
         if ev: ev[4].record()
-        return ps
+        return lambda: tq.tq_decompress_aggregate_device_params(packed, d, params_dev, w.num_levels, out=out)
 
     def barrier():
         if world > 1:
@@ -270,6 +285,7 @@ def main():
 
     # per-kernel durations inside the timed region (CUDA events on the launching stream)
     t_stats = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)       # two launches
+    t_params = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)      # device kernel, or copy + sync + host design
     t_comp = statistics.mean(e[2].elapsed_time(e[3]) for e in evs)
     t_dec = statistics.mean(e[3].elapsed_time(e[4]) for e in evs)
     peak, peak_kind = hbm_peak()
@@ -278,18 +294,19 @@ def main():
         "tq_compress": (N * d * esz + N * d * bits // 8, t_comp, 1),
         "tq_decompress_aggregate": (N * d * bits // 8 + 4 * d, t_dec, 1),
     }
-    kernels = {k: {"ms": t, "launches_per_step": n, "algorithmic_bytes": b, "gbs": b / (t * 1e-3) / 1e9,
-                   "frac_of_hbm_peak": b / (t * 1e-3) / 1e9 / peak} for k, (b, t, n) in alg.items()}
+    kernels = {"tq_params": {"ms": t_params, "where": "host (one sync)" if args.host_params else "device kernel"}}
+    kernels.update({k: {"ms": t, "launches_per_step": n, "algorithmic_bytes": b, "gbs": b / (t * 1e-3) / 1e9,
+                   "frac_of_hbm_peak": b / (t * 1e-3) / 1e9 / peak} for k, (b, t, n) in alg.items()})
 
     # decompress-aggregate again with the packed rows evicted from L2 first (in the round above they
     # were just written by tq_compress, so part of them is still cache-resident)
-    ps = one_round()
+    decompress_again = one_round()
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
     cold = []
     for _ in range(5):
         flush.fill_(1)
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(); tq.tq_decompress_aggregate(packed, d, ps, out=out); b.record()
+        a.record(); decompress_again(); b.record()
         torch.cuda.synchronize()
         cold.append(a.elapsed_time(b))
     t_cold = statistics.mean(cold)
@@ -317,11 +334,16 @@ def main():
         def e2e_round():
             g2.copy_(host_g, non_blocking=True)
             tq.tq_stats(g2, d, stats_dev=stats_dev, workspace=ws)
-            stats_pin.copy_(stats_dev, non_blocking=True)
-            stream.synchronize()
-            pp = tq.tq_params_batch(stats_pin, N, w.num_levels, mode, w.gamma)
-            tq.tq_compress(g2, pp, seed=1234, d=d, packed=packed)
-            tq.tq_decompress_aggregate(packed, d, pp, out=out)
+            if args.host_params:
+                stats_pin.copy_(stats_dev, non_blocking=True)
+                stream.synchronize()
+                pp = tq.tq_params_batch(stats_pin, N, w.num_levels, mode, w.gamma)
+                tq.tq_compress(g2, pp, seed=1234, d=d, packed=packed)
+                tq.tq_decompress_aggregate(packed, d, pp, out=out)
+            else:
+                tq.tq_params_device(stats_dev, N, w.num_levels, mode, w.gamma, params_dev=params_dev)
+                tq.tq_compress_device_params(g2, params_dev, w.num_levels, mode, seed=1234, d=d, packed=packed)
+                tq.tq_decompress_aggregate_device_params(packed, d, params_dev, w.num_levels, out=out)
             host_out.copy_(out, non_blocking=True)
 
         e2e_round(); barrier()
@@ -353,6 +375,7 @@ def main():
             "config": {"workload": w.name, "d": d, "n_workers": N, "mode": w.mode, "levels": w.num_levels, "bits": bits,
                        "gamma": w.gamma, "scale": w.scale, "storage": str(w.dtype).split(".")[-1],
                        "g_min": "mean|g| per worker (two statistics passes)", "alpha_rule": "fixed point",
+                       "params": "host" if args.host_params else "device (no host round trip inside the round)",
                        "l2": f"inputs ({in_bytes / 1e6:.0f} MB) exceed L2; packed rows ({N * words * 4 / 1e6:.0f} MB) are "
                              "re-read right after being written, see kernels.tq_decompress_aggregate.cold_l2_*",
                        "multi_gpu": "independent replica per rank, no data-path collective"},

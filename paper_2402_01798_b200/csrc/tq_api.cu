@@ -159,7 +159,7 @@ tq_status tq_compress_device_params(const void* grad_dev, tq_dtype dtype, uint64
                        static_cast<cudaStream_t>(stream)};
     const cudaError_t e = tq::launch_compress(c);
     if (e != cudaSuccess) return cuda_failed(e);
-    g_launches += 1;
+    g_launches += mode == TQ_NONUNIFORM ? 2 : 1;     // table mode: main kernel + the (usually empty) binary-search pass
     return TQ_OK;
 }
 

@@ -329,36 +329,21 @@ compress_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
                                        packed, words_stride, words_out);
 }
 
-// Out-of-line copy of the binary-search block for the run-time fallback of compress_kernel_dev, so
-// that the rarely taken path does not compete for registers with the grid path.
-template <int BITS, bool BF16>
-__device__ __noinline__ void compress_block_binary(const WorkerQ& q, float2* s_grid, float2* s_cell, float* s_search,
-                                                   const void* grad, uint64_t d, uint64_t grad_stride, const RoundKeys& rk,
-                                                   uint32_t worker, uint32_t wi, uint32_t* packed, uint64_t words_stride,
-                                                   uint64_t words_out) {
-    compress_block<BITS, kBinary, BF16>(q, s_grid, s_cell, s_search, grad, d, grad_stride, rk, worker, wi, packed,
-                                        words_stride, words_out);
-}
-
 // The grid cell of a value as a plain integer (device copy of the host's cell_of).
 __device__ __forceinline__ uint32_t cell_index(float g, float alpha, float inv_2alpha, uint32_t cells) {
-    return __float_as_uint(grid_cell(g, alpha, inv_2alpha, ldexpf(static_cast<float>(cells), -149)));
+    return __float_as_uint(grid_cell(g, alpha, inv_2alpha, __uint_as_float(cells)));   // M * 2^-149 has bit pattern M
 }
 
 // Quantizers read from device memory (tq_params_device): no host round trip before the launch.
 // Thread 0 turns worker wi's tq_params_t into the kernel's WorkerQ, including the choice of the lookup
-// grid; a worker marked invalid (alpha = 0) gets an all-zero row.  NONUNIFORM: the grid search, or the
-// binary search when no grid separates the levels, chosen per block at run time.
-template <int BITS, bool NONUNIFORM, bool BF16>
-__global__ void __launch_bounds__(kThreads, TQ_COMPRESS_MIN_BLOCKS)
-compress_kernel_dev(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
-                    const tq_params_t* __restrict__ params, const __grid_constant__ RoundKeys rk,
-                    uint32_t first_worker, uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_out) {
-    __shared__ __align__(16) float2 s_grid[NONUNIFORM ? kMaxGridCells + 1 : 1];
-    __shared__ __align__(16) float2 s_cell[TQ_MAX_LEVELS];
-    __shared__ float s_search[2 * TQ_MAX_LEVELS];
-    __shared__ WorkerQ s_q;
-    const uint32_t wi = blockIdx.y;
+// grid.  Returns false when this block has nothing to do in a kernel of kind FALLBACK:
+//   FALLBACK = false (main kernel): uniform rows, rows with a lookup grid, and all-zero rows for workers
+//              marked invalid (alpha = 0);
+//   FALLBACK = true: only the rows whose levels no grid separates (binary search).  It is launched
+//              after the main kernel and its blocks return at once for every other row, so the rarely
+//              needed path costs one near-empty launch instead of registers in the main kernel.
+template <int BITS, bool NONUNIFORM>
+__device__ __forceinline__ void load_worker(const tq_params_t* __restrict__ params, uint32_t wi, WorkerQ& s_q) {
     if (threadIdx.x < TQ_MAX_LEVELS) {
         s_q.levels[threadIdx.x] = params[wi].levels[threadIdx.x];
         s_q.inv_width[threadIdx.x] = params[wi].inv_width[threadIdx.x];
@@ -381,9 +366,22 @@ compress_kernel_dev(const void* __restrict__ grad, uint64_t d, uint64_t grad_str
             }
         }
         s_q.cells = cells;
-        s_q.cell_scale = ldexpf(static_cast<float>(cells), -149);
+        s_q.cell_scale = __uint_as_float(cells);
     }
     __syncthreads();
+}
+
+template <int BITS, bool NONUNIFORM, bool BF16>
+__global__ void __launch_bounds__(kThreads, TQ_COMPRESS_MIN_BLOCKS)
+compress_kernel_dev(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
+                    const tq_params_t* __restrict__ params, const __grid_constant__ RoundKeys rk,
+                    uint32_t first_worker, uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_out) {
+    __shared__ __align__(16) float2 s_grid[NONUNIFORM ? kMaxGridCells + 1 : 1];
+    __shared__ __align__(16) float2 s_cell[TQ_MAX_LEVELS];
+    __shared__ float s_search[2 * TQ_MAX_LEVELS];
+    __shared__ WorkerQ s_q;
+    const uint32_t wi = blockIdx.y;
+    load_worker<BITS, NONUNIFORM>(params, wi, s_q);
     if (!(s_q.alpha > 0.0f)) {       // invalid parameters: the row is all code 0
         uint32_t* prow = packed + static_cast<uint64_t>(wi) * words_stride;
         for (uint64_t w = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x; w < words_out;
@@ -391,17 +389,27 @@ compress_kernel_dev(const void* __restrict__ grad, uint64_t d, uint64_t grad_str
             prow[w] = 0u;
         return;
     }
-    if constexpr (!NONUNIFORM) {
-        compress_block<BITS, kUniform, BF16>(s_q, s_grid, s_cell, s_search, grad, d, grad_stride, rk, first_worker + wi, wi,
-                                             packed, words_stride, words_out);
-    } else {
-        if (s_q.cells != 0)
-            compress_block<BITS, kGrid, BF16>(s_q, s_grid, s_cell, s_search, grad, d, grad_stride, rk, first_worker + wi, wi,
-                                              packed, words_stride, words_out);
-        else
-            compress_block_binary<BITS, BF16>(s_q, s_grid, s_cell, s_search, grad, d, grad_stride, rk, first_worker + wi, wi,
-                                              packed, words_stride, words_out);
+    if constexpr (NONUNIFORM) {
+        if (s_q.cells == 0) return;  // left to compress_kernel_dev_fallback
     }
+    compress_block<BITS, NONUNIFORM ? kGrid : kUniform, BF16>(s_q, s_grid, s_cell, s_search, grad, d, grad_stride, rk,
+                                                              first_worker + wi, wi, packed, words_stride, words_out);
+}
+
+template <int BITS, bool BF16>
+__global__ void __launch_bounds__(kThreads, TQ_COMPRESS_MIN_BLOCKS)
+compress_kernel_dev_fallback(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
+                             const tq_params_t* __restrict__ params, const __grid_constant__ RoundKeys rk,
+                             uint32_t first_worker, uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_out) {
+    __shared__ __align__(16) float2 s_grid[1];
+    __shared__ __align__(16) float2 s_cell[TQ_MAX_LEVELS];
+    __shared__ float s_search[2 * TQ_MAX_LEVELS];
+    __shared__ WorkerQ s_q;
+    const uint32_t wi = blockIdx.y;
+    load_worker<BITS, true>(params, wi, s_q);
+    if (!(s_q.alpha > 0.0f) || s_q.cells != 0) return;
+    compress_block<BITS, kBinary, BF16>(s_q, s_grid, s_cell, s_search, grad, d, grad_stride, rk, first_worker + wi, wi,
+                                        packed, words_stride, words_out);
 }
 
 // ---- host side ---------------------------------------------------------------------------------------
@@ -491,8 +499,16 @@ cudaError_t launch_compress(const CompressCall& c) {
 
 template <int BITS, bool NU, bool BF>
 static cudaError_t launch_dev(const CompressCall& c, dim3 grid) {
+    const RoundKeys rk = round_keys(c.seed);
     compress_kernel_dev<BITS, NU, BF><<<grid, kThreads, 0, c.stream>>>(
-        c.grad, c.d, c.grad_stride, c.params_dev, round_keys(c.seed), c.first_worker, c.packed, c.words_stride, c.words_out);
+        c.grad, c.d, c.grad_stride, c.params_dev, rk, c.first_worker, c.packed, c.words_stride, c.words_out);
+    if constexpr (NU) {
+        if (cudaError_t e = cudaGetLastError()) return e;
+        // a small grid: this pass is empty unless a codebook is too crowded for the lookup grid
+        const dim3 small(grid.x < 16 ? grid.x : 16, grid.y);
+        compress_kernel_dev_fallback<BITS, BF><<<small, kThreads, 0, c.stream>>>(
+            c.grad, c.d, c.grad_stride, c.params_dev, rk, c.first_worker, c.packed, c.words_stride, c.words_out);
+    }
     return cudaGetLastError();
 }
 template <int BITS>
