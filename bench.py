@@ -3,8 +3,8 @@
 
 A step is one full round over one batch of synthetic heavy-tailed gradients already resident in
 HBM: statistics (two passes: moments, then the tail beyond g_min = mean|g|) -> closed-form
-parameters (on the device by default; --host-params copies the records back and designs them on the
-host) -> fused truncate + stochastic round + pack for all N workers -> fused unpack + dequantize +
+parameters (the 64-byte records are copied back and designed on the host: one sync per round;
+--device-params designs them on the device instead, with no host round trip) -> fused truncate + stochastic round + pack for all N workers -> fused unpack + dequantize +
 average.  Throughput is bytes of gradient input (N * d * elemsize) per
 second of step time.
 
@@ -185,11 +185,12 @@ def main():
     ap.add_argument("--variant", type=int, default=None,
                     help="with --config 3: index 0..11 into the bf16 sweep (gamma x mode x levels)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--host-params", action="store_true",
-                    help="design the parameters on the host (statistics copied back, one sync per round)")
+    ap.add_argument("--device-params", action="store_true",
+                    help="design the parameters on the device (tq_params_device): no host round trip inside the round")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
+    args.host_params = not args.device_params
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     from paper_2402_01798_b200 import inputs
@@ -245,7 +246,7 @@ def main():
             tq.tq_decompress_aggregate(packed, d, ps, out=out)
             if ev: ev[4].record()
             return lambda: tq.tq_decompress_aggregate(packed, d, ps, out=out)
-        # default: parameters designed on the device, nothing returns to the host inside the round
+        # --device-params: parameters designed on the device, nothing returns to the host inside the round
         tq.tq_params_device(stats_dev, N, w.num_levels, mode, w.gamma, params_dev=params_dev)
         if ev: ev[2].record()
         tq.tq_compress_device_params(g, params_dev, w.num_levels, mode, seed=1234, d=d, packed=packed)

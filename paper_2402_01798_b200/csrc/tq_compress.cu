@@ -348,20 +348,28 @@ __device__ __forceinline__ void load_worker(const tq_params_t* __restrict__ para
         s_q.levels[threadIdx.x] = params[wi].levels[threadIdx.x];
         s_q.inv_width[threadIdx.x] = params[wi].inv_width[threadIdx.x];
     }
+    __syncthreads();                 // the levels are in shared memory from here on
     if (threadIdx.x == 0) {
         const tq_params_t& p = params[wi];
-        const bool ok = p.alpha > 0.0f && p.bits == BITS && !(p.flags & TQ_FLAG_INVALID);
-        s_q.alpha = ok ? p.alpha : 0.0f;
+        const float alpha = p.alpha;
+        const bool ok = alpha > 0.0f && p.bits == BITS && !(p.flags & TQ_FLAG_INVALID);
+        const float inv_2alpha = ok ? __fdiv_rn(1.0f, __fmul_rn(2.0f, alpha)) : 0.0f;
+        s_q.alpha = ok ? alpha : 0.0f;
         s_q.inv_step = p.inv_step;
         s_q.top = static_cast<float>((1 << BITS) - 1);
-        s_q.inv_2alpha = ok ? __fdiv_rn(1.0f, __fmul_rn(2.0f, p.alpha)) : 0.0f;
+        s_q.inv_2alpha = inv_2alpha;
         uint32_t cells = 0;
-        if (NONUNIFORM && ok && s_q.inv_2alpha <= 3.402823466e38f) {
+        if (NONUNIFORM && ok && inv_2alpha <= 3.402823466e38f) {
             constexpr int s = (1 << BITS) - 1;
             for (uint32_t m = kMinGridCells; m <= static_cast<uint32_t>(kMaxGridCells) && cells == 0; m *= 2) {
                 bool distinct = true;
-                for (int j = 2; j <= s - 1 && distinct; ++j)
-                    distinct = cell_index(p.levels[j], p.alpha, s_q.inv_2alpha, m) > cell_index(p.levels[j - 1], p.alpha, s_q.inv_2alpha, m);
+                uint32_t prev = s >= 2 ? cell_index(s_q.levels[1], alpha, inv_2alpha, m) : 0u;
+#pragma unroll
+                for (int j = 2; j <= s - 1; ++j) {
+                    const uint32_t cur = cell_index(s_q.levels[j], alpha, inv_2alpha, m);
+                    distinct = distinct && cur > prev;
+                    prev = cur;
+                }
                 if (distinct) cells = m;
             }
         }
