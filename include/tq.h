@@ -50,11 +50,16 @@ typedef enum {
 } tq_status;
 
 typedef enum { TQ_F32 = 0, TQ_BF16 = 1 } tq_dtype;               /* gradient storage type */
-typedef enum { TQ_UNIFORM = 0, TQ_NONUNIFORM = 1 } tq_mode;
+typedef enum {
+    TQ_UNIFORM = 0,     /* evenly spaced levels (Section 4.1) */
+    TQ_NONUNIFORM = 1,  /* density proportional to p^(1/3) (Section 4.2); also any caller-made codebook */
+    TQ_BISCALED = 2     /* two step sizes, inside and outside k* alpha (Appendix, truncated BiScaled) */
+} tq_mode;
 typedef enum {
     TQ_ALPHA_CLOSED = 0,       /* alpha' : the boxed equation with Q = 1 (text after Theorem 1) */
     TQ_ALPHA_FIXED_POINT = 1,  /* iterate the boxed equation of Section 4.1 / 4.2 */
-    TQ_ALPHA_USER = 2          /* caller supplies alpha */
+    TQ_ALPHA_USER = 2,         /* caller supplies alpha */
+    TQ_ALPHA_MAXABS = 3        /* alpha = max|g|: no truncation (the QSGD / NQSGD baselines of Section 5) */
 } tq_alpha_rule;
 
 enum { TQ_FLAG_ALPHA_CAPPED = 1, TQ_FLAG_ALPHA_AT_GMIN = 2, TQ_FLAG_GAMMA_FROM_MLE = 4,
@@ -153,9 +158,14 @@ tq_status tq_stats_static(const void* grad_dev, tq_dtype dtype, uint64_t d, uint
  *                relative change is <= 1e-12 or 10000 iterations.  Both are clamped to
  *                [g_min, max_abs] (flags ALPHA_AT_GMIN / ALPHA_CAPPED).
  *                USER: alpha_user, unclamped.
+ *                MAXABS: alpha = max_abs, so nothing is truncated: with UNIFORM this is the paper's QSGD
+ *                baseline, with NONUNIFORM its NQSGD baseline (Section 5).
  *   mode         UNIFORM: l_k = -alpha + k 2 alpha / s.  NONUNIFORM: the boxed density
  *                lambda_s proportional to p^(1/3) (Section 4.2), turned into levels by
- *                integral_{-alpha}^{l_k} lambda_s = k.
+ *                integral_{-alpha}^{l_k} lambda_s = k.  BISCALED: the Appendix's two-piece density
+ *                (k* = argmin_k Q_B(alpha, k) by a 65-point scan + golden section, alpha from the
+ *                boxed BiScaled equation with k* recomputed at every step), levels by the same rule.
+ *                To the kernels BISCALED is a table codebook like NONUNIFORM.
  * Errors: INVALID_ARG, DOMAIN, DEGENERATE_LEVELS.  out_host is unspecified on error.
  */
 tq_status tq_params(const tq_stats_t* stats_host, uint32_t num_levels, tq_mode mode, double gamma,

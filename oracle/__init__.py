@@ -24,8 +24,8 @@ _SRC = os.path.join(_HERE, "tq_oracle.c")
 _LIB = os.path.join(_HERE, "libtq_oracle.so")
 
 MAX_LEVELS = 16
-UNIFORM, NONUNIFORM = 0, 1
-ALPHA_CLOSED, ALPHA_FIXED_POINT, ALPHA_USER = 0, 1, 2
+UNIFORM, NONUNIFORM, BISCALED = 0, 1, 2
+ALPHA_CLOSED, ALPHA_FIXED_POINT, ALPHA_USER, ALPHA_MAXABS = 0, 1, 2, 3
 FLAG_ALPHA_CAPPED, FLAG_ALPHA_AT_GMIN, FLAG_GAMMA_FROM_MLE = 1, 2, 4
 OK, ERR_ARG, ERR_DOMAIN, ERR_LEVELS = 0, -1, -2, -5
 
@@ -85,8 +85,10 @@ def lib() -> C.CDLL:
         for name in ("orc_model_pdf", "orc_model_QU", "orc_model_H", "orc_model_Hinv",
                      "orc_model_QN", "orc_truncation_bias"):
             fn = getattr(L, name); fn.argtypes = [P(Model), f64]; fn.restype = f64
-        for name in ("orc_etq_uniform", "orc_etq_nonuniform", "orc_etq_theorem"):
+        for name in ("orc_etq_uniform", "orc_etq_nonuniform", "orc_etq_theorem", "orc_etq_biscaled", "orc_model_QB"):
             fn = getattr(L, name); fn.argtypes = [P(Model), f64, f64]; fn.restype = f64
+        L.orc_biscaled_kstar.argtypes = [P(Model), f64]; L.orc_biscaled_kstar.restype = f64
+        L.orc_biscaled_density.argtypes = [P(Model), f64, f64, P(f64), P(f64), P(f64)]; L.orc_biscaled_density.restype = None
         L.orc_alpha_prime.argtypes = [P(Model), f64]; L.orc_alpha_prime.restype = f64
         L.orc_alpha_fixed_point.argtypes = [P(Model), f64, i32, f64, P(i32), P(i32)]
         L.orc_alpha_fixed_point.restype = f64
@@ -187,6 +189,17 @@ def table_params(levels: Sequence[float], mode: int = NONUNIFORM) -> Params:
 def model_fn(name: str, model: Model, x: float, s: Optional[float] = None) -> float:
     fn = getattr(lib(), "orc_" + name)
     return float(fn(C.byref(model), x) if s is None else fn(C.byref(model), x, s))
+
+
+def biscaled_kstar(model: Model, alpha: float) -> float:
+    return float(lib().orc_biscaled_kstar(C.byref(model), alpha))
+
+
+def biscaled_density(model: Model, alpha: float, s: float):
+    """(k*, lambda_in, lambda_out) of the boxed BiScaled density."""
+    k, a, b = C.c_double(), C.c_double(), C.c_double()
+    lib().orc_biscaled_density(C.byref(model), alpha, s, C.byref(k), C.byref(a), C.byref(b))
+    return k.value, a.value, b.value
 
 
 def alpha_prime(model: Model, s: float) -> float:

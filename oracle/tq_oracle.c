@@ -24,6 +24,7 @@
  *   lambda_s proportional to p^(1/3) (boxed) .. Section 4.2, boxed density
  *   Q_N(alpha), alpha non-uniform (boxed) ..... Section 4.2
  *   gamma maximum-likelihood estimate ......... Section 5, experimental setting
+ *   BiScaled density, Q_B, alpha (boxed) ...... Appendix, "Truncated BiScaled Quantization"
  *   server aggregation ........................ Algorithm 1, server step; Lemma 2 (w_i = 1/N)
  *
  * What the paper leaves open is fixed here (one reading each, listed for the reader):
@@ -49,6 +50,12 @@
  *       probability >= 1 and always receives code s (Section 3.1: |g| > alpha maps to
  *       sgn(g) alpha, which is a codebook point).
  *   R12 wire format: dense LSB-first bit stream over little-endian 32-bit words, pad zero.
+ *   R16 the no-truncation baselines of Section 5 (QSGD, NQSGD) are the same quantizers with
+ *       alpha = max|g| (alpha rule MAXABS), so that the truncation operator is the identity.
+ *   R17 truncated BiScaled quantizer (Appendix): k* = argmin_k Q_B(alpha, k) is found by a scan of
+ *       k = j/64 followed by 60 golden-section steps in the bracketing pair of cells; alpha iterates the
+ *       boxed BiScaled equation as in R8 with k* recomputed at every step; s_alpha, s_beta are real
+ *       numbers (the Appendix's formulas), so the levels come from the two-piece density by R7.
  *   R13 aggregation: fp32 adds in worker order, then one IEEE division by N; with
  *       weights, each product w_i * v_i is rounded, then added, no division.
  */
@@ -59,8 +66,8 @@
 #define ORC_MAX_LEVELS 16
 
 enum { ORC_OK = 0, ORC_ERR_ARG = -1, ORC_ERR_DOMAIN = -2, ORC_ERR_LEVELS = -5 };
-enum { ORC_UNIFORM = 0, ORC_NONUNIFORM = 1 };
-enum { ORC_ALPHA_CLOSED = 0, ORC_ALPHA_FIXED_POINT = 1, ORC_ALPHA_USER = 2 };
+enum { ORC_UNIFORM = 0, ORC_NONUNIFORM = 1, ORC_BISCALED = 2 };
+enum { ORC_ALPHA_CLOSED = 0, ORC_ALPHA_FIXED_POINT = 1, ORC_ALPHA_USER = 2, ORC_ALPHA_MAXABS = 3 };
 enum { ORC_FLAG_ALPHA_CAPPED = 1, ORC_FLAG_ALPHA_AT_GMIN = 2, ORC_FLAG_GAMMA_FROM_MLE = 4 };
 
 /* ------------------------------------------------------------------------------------ */
@@ -208,6 +215,48 @@ double orc_model_QN(const orc_model_t *m, double alpha)
     return 2.0 * h * h * h / (alpha * alpha);
 }
 
+/* Appendix: Q_B(alpha, k) = [ (2 int_{k alpha}^{alpha} p)^(1/3) (1-k)^(2/3) + (2 int_0^{k alpha} p)^(1/3) k^(2/3) ]^3 */
+double orc_model_QB(const orc_model_t *m, double alpha, double k)
+{
+    double inner = orc_model_QU(m, k * alpha);               /* 2 int_0^{k alpha} p */
+    double outer = orc_model_QU(m, alpha) - inner;           /* 2 int_{k alpha}^{alpha} p */
+    if (outer < 0.0) outer = 0.0;
+    double t = cbrt(outer) * pow(1.0 - k, 2.0 / 3.0) + cbrt(inner) * pow(k, 2.0 / 3.0);
+    return t * t * t;
+}
+
+/* R17: k* = argmin_k Q_B(alpha, k) on [0, 1]. */
+double orc_biscaled_kstar(const orc_model_t *m, double alpha)
+{
+    int best = 0;
+    double best_q = orc_model_QB(m, alpha, 0.0);
+    for (int j = 1; j <= 64; ++j) {
+        double q = orc_model_QB(m, alpha, (double)j / 64.0);
+        if (q < best_q) { best_q = q; best = j; }
+    }
+    double lo = (best > 0 ? best - 1 : 0) / 64.0, hi = (best < 64 ? best + 1 : 64) / 64.0;
+    const double r = 0.6180339887498949;                     /* (sqrt 5 - 1) / 2 */
+    double x1 = hi - r * (hi - lo), x2 = lo + r * (hi - lo);
+    double f1 = orc_model_QB(m, alpha, x1), f2 = orc_model_QB(m, alpha, x2);
+    for (int it = 0; it < 60; ++it) {
+        if (f1 <= f2) { hi = x2; x2 = x1; f2 = f1; x1 = hi - r * (hi - lo); f1 = orc_model_QB(m, alpha, x1); }
+        else          { lo = x1; x1 = x2; f1 = f2; x2 = lo + r * (hi - lo); f2 = orc_model_QB(m, alpha, x2); }
+    }
+    return 0.5 * (lo + hi);
+}
+
+/* The boxed BiScaled density: lambda_in on |g| <= k* alpha, lambda_out on k* alpha < |g| <= alpha. */
+void orc_biscaled_density(const orc_model_t *m, double alpha, double s, double *k_out, double *lam_in, double *lam_out)
+{
+    double k = orc_biscaled_kstar(m, alpha);
+    double beta = k * alpha;
+    double p1 = orc_model_QU(m, beta) / (2.0 * beta);                              /* mean density on [0, beta] */
+    double p2 = (orc_model_QU(m, alpha) - orc_model_QU(m, beta)) / (2.0 * (alpha - beta));
+    double c1 = cbrt(p1), c2 = cbrt(p2);
+    double denom = 2.0 * c2 * (1.0 - k) * alpha + 2.0 * c1 * k * alpha;
+    *k_out = k; *lam_in = c1 * s / denom; *lam_out = c2 * s / denom;
+}
+
 /* Truncation-bias term of the error equations, per element and per 1/N:
  * 4 rho g_min^(gamma-1) alpha^(3-gamma) / ((gamma-2)(gamma-3)); needs gamma > 3, alpha >= g_min. */
 double orc_truncation_bias(const orc_model_t *m, double alpha)
@@ -229,6 +278,12 @@ double orc_etq_nonuniform(const orc_model_t *m, double alpha, double s)
     return orc_model_QN(m, alpha) * alpha * alpha / (s * s) + orc_truncation_bias(m, alpha);
 }
 
+/* E_TQ(alpha, k*) * N / d for the BiScaled density (Appendix error equation). */
+double orc_etq_biscaled(const orc_model_t *m, double alpha, double s)
+{
+    return orc_model_QB(m, alpha, orc_biscaled_kstar(m, alpha)) * alpha * alpha / (s * s) + orc_truncation_bias(m, alpha);
+}
+
 /* Theorems 1 and 2: the error term at the optimum, given Q = Q_U(alpha*) or Q_N(alpha*). */
 double orc_etq_theorem(const orc_model_t *m, double Q, double s)
 {
@@ -247,7 +302,9 @@ double orc_alpha_prime(const orc_model_t *m, double s)
 /* One application of the boxed equation's right-hand side. */
 static double alpha_map(const orc_model_t *m, double s, int mode, double alpha)
 {
-    double Q = (mode == ORC_UNIFORM) ? orc_model_QU(m, alpha) : orc_model_QN(m, alpha);
+    double Q = (mode == ORC_UNIFORM) ? orc_model_QU(m, alpha)
+             : (mode == ORC_NONUNIFORM) ? orc_model_QN(m, alpha)
+             : orc_model_QB(m, alpha, orc_biscaled_kstar(m, alpha));
     return m->g_min * pow(2.0 * m->rho * s * s / ((m->gamma - 2.0) * Q), 1.0 / (m->gamma - 1.0));
 }
 
@@ -313,6 +370,19 @@ int orc_build_table(const orc_model_t *m, uint32_t num_levels, int mode, float a
         /* Section 4.1: l_k = -alpha + k * 2 alpha / s */
         for (uint32_t k = 0; k <= s; ++k)
             p->levels[k] = (float)(-a + (double)k * (2.0 * a / (double)s));
+    } else if (mode == ORC_BISCALED) {
+        /* R17 + R7: cumulative density from the centre reaches k - s/2 at level k */
+        double kk, lam_in, lam_out;
+        orc_biscaled_density(m, a, (double)s, &kk, &lam_in, &lam_out);
+        double beta = kk * a;
+        for (uint32_t k = 0; k <= s; ++k) {
+            if (2 * k < s) continue;
+            double c = (double)k - 0.5 * (double)s;
+            double x = (c <= lam_in * beta) ? c / lam_in : beta + (c - lam_in * beta) / lam_out;
+            float l = (float)x;
+            p->levels[k] = l;
+            p->levels[s - k] = -l;
+        }
     } else {
         /* R7: H(l_k) = (2k/s - 1) H(alpha); upper half computed, lower half mirrored */
         double Ha = orc_model_H(m, a);
@@ -350,7 +420,7 @@ int orc_params(const orc_stats_t *st, uint32_t num_levels, int mode, double gamm
     uint32_t bits = 0;
     while (bits < 5 && (1u << bits) != num_levels) ++bits;
     if (bits < 1 || bits > 4) return ORC_ERR_ARG;
-    if (mode != ORC_UNIFORM && mode != ORC_NONUNIFORM) return ORC_ERR_ARG;
+    if (mode != ORC_UNIFORM && mode != ORC_NONUNIFORM && mode != ORC_BISCALED) return ORC_ERR_ARG;
     p->bits = bits; p->num_levels = num_levels; p->mode = (uint32_t)mode;
     double s = (double)(num_levels - 1);
 
@@ -370,6 +440,10 @@ int orc_params(const orc_stats_t *st, uint32_t num_levels, int mode, double gamm
     if (alpha_rule == ORC_ALPHA_USER) {
         if (!(alpha_user > 0.0) || !isfinite(alpha_user)) return ORC_ERR_DOMAIN;
         alpha = alpha_user;
+    } else if (alpha_rule == ORC_ALPHA_MAXABS) {
+        /* Section 5 baselines QSGD / NQSGD: quantization without truncation, the range is max|g| */
+        if (!(st->max_abs > 0.0f)) return ORC_ERR_DOMAIN;
+        alpha = (double)st->max_abs;
     } else {
         double cap = (double)st->max_abs;
         int capped = 0, iters = 0;

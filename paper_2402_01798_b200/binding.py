@@ -21,8 +21,8 @@ OK, ERR_INVALID_ARG, ERR_DOMAIN, ERR_ALIGNMENT, ERR_BUFFER_TOO_SMALL, ERR_DEGENE
 ERR_STATIC_LIMIT = -7
 STATIC_MAX_WORKERS = 16
 F32, BF16 = 0, 1
-UNIFORM, NONUNIFORM = 0, 1
-ALPHA_CLOSED, ALPHA_FIXED_POINT, ALPHA_USER = 0, 1, 2
+UNIFORM, NONUNIFORM, BISCALED = 0, 1, 2
+ALPHA_CLOSED, ALPHA_FIXED_POINT, ALPHA_USER, ALPHA_MAXABS = 0, 1, 2, 3
 FLAG_ALPHA_CAPPED, FLAG_ALPHA_AT_GMIN, FLAG_GAMMA_FROM_MLE, FLAG_INVALID = 1, 2, 4, 8
 
 EXPORTS = ("tq_packed_words", "tq_stats_workspace_bytes", "tq_stats", "tq_stats_static", "tq_params", "tq_params_batch", "tq_params_from_levels", "tq_params_device",

@@ -35,7 +35,7 @@ tq_status check_params(const tq_params_t* p, uint32_t n, uint32_t* bits) {
     if (b < 1 || b > 4) return TQ_ERR_INVALID_ARG;
     for (uint32_t i = 0; i < n; ++i) {
         if (p[i].bits != b || p[i].num_levels != (1u << b)) return TQ_ERR_INVALID_ARG;
-        if (p[i].mode != TQ_UNIFORM && p[i].mode != TQ_NONUNIFORM) return TQ_ERR_INVALID_ARG;
+        if (p[i].mode != TQ_UNIFORM && p[i].mode != TQ_NONUNIFORM && p[i].mode != TQ_BISCALED) return TQ_ERR_INVALID_ARG;
         if (!(p[i].alpha > 0.0f)) return TQ_ERR_DOMAIN;
     }
     *bits = b;
@@ -92,15 +92,15 @@ tq_status tq_compress(const void* grad_dev, tq_dtype dtype, uint64_t d, uint64_t
     if (tq_status s = check_grad(grad_dev, dtype, d, grad_stride, n_workers)) return s;
     uint32_t bits = 0;
     if (tq_status s = check_params(params_host, n_workers, &bits)) return s;
-    for (uint32_t i = 1; i < n_workers; ++i)
-        if (params_host[i].mode != params_host[0].mode) return TQ_ERR_INVALID_ARG;
+    for (uint32_t i = 1; i < n_workers; ++i)      // one kernel per launch: all uniform, or all table codebooks
+        if ((params_host[i].mode == TQ_UNIFORM) != (params_host[0].mode == TQ_UNIFORM)) return TQ_ERR_INVALID_ARG;
     const size_t need = tq_packed_words(d, bits);
     if (need && !packed_dev) return TQ_ERR_INVALID_ARG;
     if (!aligned(packed_dev, 16) || words_stride % 4 != 0) return TQ_ERR_ALIGNMENT;
     if (words_stride < need) return TQ_ERR_BUFFER_TOO_SMALL;
     if (d == 0) return TQ_OK;
     tq::CompressCall c{grad_dev, dtype == TQ_BF16, d, grad_stride, n_workers, params_host, nullptr, bits,
-                       params_host[0].mode == TQ_NONUNIFORM, seed, first_worker, packed_dev, words_stride, need,
+                       params_host[0].mode != TQ_UNIFORM, seed, first_worker, packed_dev, words_stride, need,
                        static_cast<cudaStream_t>(stream)};
     const cudaError_t e = tq::launch_compress(c);
     if (e != cudaSuccess) return cuda_failed(e);
@@ -155,11 +155,11 @@ tq_status tq_compress_device_params(const void* grad_dev, tq_dtype dtype, uint64
     if (words_stride < need) return TQ_ERR_BUFFER_TOO_SMALL;
     if (d == 0) return TQ_OK;
     tq::CompressCall c{grad_dev, dtype == TQ_BF16, d, grad_stride, n_workers, nullptr, params_dev, bits,
-                       mode == TQ_NONUNIFORM, seed, first_worker, packed_dev, words_stride, need,
+                       mode != TQ_UNIFORM, seed, first_worker, packed_dev, words_stride, need,
                        static_cast<cudaStream_t>(stream)};
     const cudaError_t e = tq::launch_compress(c);
     if (e != cudaSuccess) return cuda_failed(e);
-    g_launches += mode == TQ_NONUNIFORM ? 2 : 1;     // table mode: main kernel + the (usually empty) binary-search pass
+    g_launches += mode != TQ_UNIFORM ? 2 : 1;     // table mode: main kernel + the (usually empty) binary-search pass
     return TQ_OK;
 }
 

@@ -58,7 +58,37 @@ struct TailModel {
         const double two_i = 2.0 * cuberoot_integral(a);
         return two_i * two_i * two_i / (4.0 * a * a);
     }
-    TQ_HD double q_of(uint32_t mode, double a) const { return mode == TQ_UNIFORM ? mass_inside(a) : holder_factor(a); }
+    // Q_B of the Appendix for the split at k * a: inner and outer mass, each spread evenly
+    TQ_HD double biscaled_factor(double a, double k) const {
+        const double inner = mass_inside(k * a);
+        double outer = mass_inside(a) - inner;
+        if (outer < 0.0) outer = 0.0;
+        const double t = cbrt(outer) * pow(1.0 - k, 2.0 / 3.0) + cbrt(inner) * pow(k, 2.0 / 3.0);
+        return t * t * t;
+    }
+    // k* = argmin_k Q_B(a, k): scan k = j/64, then 60 golden-section steps between the neighbours of the best j
+    TQ_HD double biscaled_split(double a) const {
+        int best = 0;
+        double best_q = biscaled_factor(a, 0.0);
+        for (int j = 1; j <= 64; ++j) {
+            const double q = biscaled_factor(a, j / 64.0);
+            if (q < best_q) { best_q = q; best = j; }
+        }
+        double lo = (best > 0 ? best - 1 : 0) / 64.0, hi = (best < 64 ? best + 1 : 64) / 64.0;
+        const double r = 0.6180339887498949;
+        double x1 = hi - r * (hi - lo), x2 = lo + r * (hi - lo);
+        double f1 = biscaled_factor(a, x1), f2 = biscaled_factor(a, x2);
+        for (int it = 0; it < 60; ++it) {
+            if (f1 <= f2) { hi = x2; x2 = x1; f2 = f1; x1 = hi - r * (hi - lo); f1 = biscaled_factor(a, x1); }
+            else { lo = x1; x1 = x2; f1 = f2; x2 = lo + r * (hi - lo); f2 = biscaled_factor(a, x2); }
+        }
+        return 0.5 * (lo + hi);
+    }
+    TQ_HD double q_of(uint32_t mode, double a) const {
+        if (mode == TQ_UNIFORM) return mass_inside(a);
+        if (mode == TQ_NONUNIFORM) return holder_factor(a);
+        return biscaled_factor(a, biscaled_split(a));
+    }
     // right-hand side of the boxed alpha equations for a given Q
     TQ_HD double alpha_for_q(double s, double q) const {
         return g_min * pow(2.0 * rho * s * s / ((gamma - 2.0) * q), 1.0 / (gamma - 1.0));
@@ -126,6 +156,9 @@ TQ_HD inline tq_status design(const tq_stats_t* st, uint32_t num_levels, uint32_
     if (rule == TQ_ALPHA_USER) {
         if (!(alpha_user > 0.0) || !finite_d(alpha_user)) return TQ_ERR_DOMAIN;
         alpha = alpha_user;
+    } else if (rule == TQ_ALPHA_MAXABS) {                    // Section 5 baselines: no truncation
+        if (!(st->max_abs > 0.0f)) return TQ_ERR_DOMAIN;
+        alpha = static_cast<double>(st->max_abs);
     } else {
         const double cap = static_cast<double>(st->max_abs);
         alpha = m.alpha_for_q(s, 1.0);                       // alpha'
@@ -169,6 +202,21 @@ TQ_HD inline tq_status design(const tq_stats_t* st, uint32_t num_levels, uint32_
     if (mode == TQ_UNIFORM) {
         const double step = 2.0 * a / s;                     // Section 4.1 codebook
         for (uint32_t k = 0; k <= si; ++k) out->levels[k] = static_cast<float>(-a + static_cast<double>(k) * step);
+    } else if (mode == TQ_BISCALED) {
+        // Appendix: density s c_in / D inside k* alpha and s c_out / D outside, c = (mean density)^(1/3),
+        // D = 2 alpha (c_out (1 - k*) + c_in k*).  Level k sits where the density accumulated from the
+        // centre reaches k - s/2.  Upper half, then mirrored.
+        const double k = m.biscaled_split(a), beta = k * a;
+        const double c_in = cbrt(m.mass_inside(beta) / (2.0 * beta));
+        const double c_out = cbrt((m.mass_inside(a) - m.mass_inside(beta)) / (2.0 * (a - beta)));
+        const double denom = 2.0 * a * (c_out * (1.0 - k) + c_in * k);
+        const double lam_in = s * c_in / denom, lam_out = s * c_out / denom;
+        for (uint32_t j = (si + 1) / 2; j <= si; ++j) {
+            const double c = static_cast<double>(j) - 0.5 * s;
+            const double x = c <= lam_in * beta ? c / lam_in : beta + (c - lam_in * beta) / lam_out;
+            out->levels[j] = static_cast<float>(x);
+            out->levels[si - j] = -static_cast<float>(x);
+        }
     } else {
         // lambda_s = s p^(1/3) / int p^(1/3): level k sits where the running integral of p^(1/3)
         // from the centre reaches (2k/s - 1) of its value at alpha.  Upper half, then mirrored.
@@ -187,8 +235,8 @@ TQ_HD inline tq_status design(const tq_stats_t* st, uint32_t num_levels, uint32_
 
 static bool valid_request(uint32_t num_levels, int mode, int rule, uint32_t* bits) {
     if (!bits_for_levels(num_levels, bits)) return false;
-    if (mode != TQ_UNIFORM && mode != TQ_NONUNIFORM) return false;
-    return rule == TQ_ALPHA_CLOSED || rule == TQ_ALPHA_FIXED_POINT || rule == TQ_ALPHA_USER;
+    if (mode != TQ_UNIFORM && mode != TQ_NONUNIFORM && mode != TQ_BISCALED) return false;
+    return rule == TQ_ALPHA_CLOSED || rule == TQ_ALPHA_FIXED_POINT || rule == TQ_ALPHA_USER || rule == TQ_ALPHA_MAXABS;
 }
 
 // One thread per worker.  A worker whose statistics are outside the model's domain gets
@@ -222,7 +270,7 @@ extern "C" tq_status tq_params_from_levels(const float* levels_host, uint32_t nu
                                            tq_params_t* out) {
     uint32_t bits = 0;
     if (!levels_host || !out || !tq::bits_for_levels(num_levels, &bits)) return TQ_ERR_INVALID_ARG;
-    if (mode != TQ_UNIFORM && mode != TQ_NONUNIFORM) return TQ_ERR_INVALID_ARG;
+    if (mode != TQ_UNIFORM && mode != TQ_NONUNIFORM && mode != TQ_BISCALED) return TQ_ERR_INVALID_ARG;
     tq::clear(out);
     out->bits = bits; out->num_levels = num_levels; out->mode = mode;
     for (uint32_t k = 0; k < num_levels; ++k) out->levels[k] = levels_host[k];

@@ -69,9 +69,9 @@ def _stats(cls, **kw):
 
 
 CASES = [(L, mode, gamma, rule)
-         for L in (2, 4, 8, 16) for mode in (0, 1)
+         for L in (2, 4, 8, 16) for mode in (0, 1, 2)
          for gamma in (2.2, 2.5, 3.0, 3.5, 4.0, 5.0, math.nan)
-         for rule in (0, 1)]
+         for rule in (0, 1, 3)]
 
 
 @pytest.mark.parametrize("L,mode,gamma,rule", CASES)

@@ -359,7 +359,8 @@ def test_config5_billion_elements_windows(tq, orc):
 
 # ----------------------------------------------------------------------- device-resident parameters
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
-@pytest.mark.parametrize("L,mode,gamma", [(4, 0, 3.0), (8, 0, 2.5), (8, 1, 2.5), (16, 1, 3.0), (16, 1, 2.2), (2, 1, 4.0), (16, 0, float("nan"))])
+@pytest.mark.parametrize("L,mode,gamma", [(4, 0, 3.0), (8, 0, 2.5), (8, 1, 2.5), (16, 1, 3.0), (16, 1, 2.2), (2, 1, 4.0), (16, 0, float("nan")),
+                                          (8, 2, 3.0), (16, 2, 2.5)])
 def test_round_without_host_round_trip(tq, orc, dtype, L, mode, gamma):
     """statistics -> tq_params_device -> tq_compress_device_params -> tq_decompress_aggregate_device_params,
     nothing copied to the host in between.  The device-made parameters agree with the host's (and so
@@ -391,6 +392,41 @@ def test_round_without_host_round_trip(tq, orc, dtype, L, mode, gamma):
     w = [0.1 * (i + 1) for i in range(n)]
     ow = tq.tq_decompress_aggregate_device_params(packed, d, params_dev, L, weights=w)
     assert torch.equal(ow, tq.tq_decompress_aggregate(packed, d, dev_ps, weights=w))
+
+
+@pytest.mark.parametrize("L", [4, 8, 16])
+def test_biscaled_codebook_through_the_table_kernels(tq, orc, L):
+    """Truncated BiScaled quantizer (Appendix): parameters from the library against the oracle's, codes
+    and aggregate bit-exact (it is a table codebook to the kernels)."""
+    d, n = 400_003, 4
+    g = heavy_tailed(d, n, torch.float32, seed=50 + L, gamma=3.5)
+    st, ps = lib_params_for(tq, g, d, L, tq.BISCALED, 3.5)
+    check_params_against_oracle(tq, orc, st, ps, L, orc.BISCALED, 3.5)
+    packed = tq.tq_compress(g, ps, seed=8, d=d)
+    out = tq.tq_decompress_aggregate(packed, d, ps)
+    ops = [to_oracle_params(orc, p) for p in ps]
+    got = packed.cpu().numpy().view(np.uint32)
+    for i in range(n):
+        assert np.array_equal(got[i], orc.compress(host_f32(orc, g[i, :d]), ops[i], 8, i))
+    assert np.array_equal(out.cpu().numpy(), orc.decompress_aggregate(got, d, ops))
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_no_truncation_baselines(tq, orc, mode):
+    """alpha = max|g| (QSGD / NQSGD of Section 5) through the same kernels, host and device parameters."""
+    d, n = 200_001, 2
+    g = heavy_tailed(d, n, torch.float32, seed=31 + mode, gamma=2.5)
+    stats_dev = tq.tq_stats(g, d)
+    st = tq.stats_to_host(stats_dev)
+    ps = [tq.tq_params(s, 8, mode, 2.5, tq.ALPHA_MAXABS) for s in st]
+    for s, p in zip(st, ps):
+        assert p.alpha == s.max_abs
+    got = tq.tq_compress(g, ps, seed=4, d=d).cpu().numpy().view(np.uint32)
+    for i in range(n):
+        assert np.array_equal(got[i], orc.compress(host_f32(orc, g[i, :d]), to_oracle_params(orc, ps[i]), 4, i))
+    pd = tq.tq_params_device(stats_dev, n, 8, mode, 2.5, tq.ALPHA_MAXABS)
+    assert [p.alpha for p in tq.params_to_host(pd)] == [p.alpha for p in ps]
+    assert torch.equal(tq.tq_compress_device_params(g, pd, 8, mode, seed=4, d=d).cpu(), torch.from_numpy(got.view(np.int32)))
 
 
 def test_device_params_marks_bad_statistics_and_fallback_codebooks(tq, orc):

@@ -33,6 +33,10 @@ MUTATIONS = [
     ("fixed-point exponent", "((m->gamma - 2.0) * Q), 1.0 / (m->gamma - 1.0))", "((m->gamma - 2.0) * Q), 1.0 / (m->gamma - 2.0))", "test_oracle_params.py"),
     ("bias denominator", "/ ((m->gamma - 2.0) * (m->gamma - 3.0));", "/ ((m->gamma - 1.0) * (m->gamma - 2.0));", "test_oracle_params.py"),
     ("level placement", "(2.0 * (double)k / (double)s - 1.0) * Ha", "((double)k / (double)s) * Ha", "test_oracle_params.py"),
+    ("biscaled exponent", "cbrt(outer) * pow(1.0 - k, 2.0 / 3.0)", "cbrt(outer) * pow(1.0 - k, 1.0 / 3.0)", "test_oracle_biscaled.py"),
+    ("biscaled density split", "double denom = 2.0 * c2 * (1.0 - k) * alpha + 2.0 * c1 * k * alpha;", "double denom = 2.0 * c2 * k * alpha + 2.0 * c1 * (1.0 - k) * alpha;", "test_oracle_biscaled.py"),
+    ("biscaled level offset", "double c = (double)k - 0.5 * (double)s;", "double c = (double)k - 0.5 * (double)(s + 1);", "test_oracle_biscaled.py"),
+    ("biscaled inner mass", "double p1 = orc_model_QU(m, beta) / (2.0 * beta);", "double p1 = orc_model_QU(m, beta) / beta;", "test_oracle_biscaled.py"),
     ("cube root dropped", "double cb = cbrt((1.0 - 2.0 * m->rho) / (2.0 * m->g_min));\n    if (x <= m->g_min) return cb * x;", "double cb = (1.0 - 2.0 * m->rho) / (2.0 * m->g_min);\n    if (x <= m->g_min) return cb * x;", "test_oracle_params.py"),
 ]
 

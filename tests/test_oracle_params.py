@@ -370,3 +370,24 @@ def test_alpha_grid_search_on_samples(orc, gamma, s):
     a_bound, a_exact = grid[e[:, 0].argmin()], grid[e[:, 1].argmin()]
     assert abs(math.log(a_bound / a_star)) < 0.10
     assert abs(math.log(a_exact / (a_star * 1.5 ** (1 / (gamma - 1))))) < 0.12
+
+
+def test_no_truncation_baselines_use_the_full_range(orc):
+    """QSGD / NQSGD of Section 5: the same quantizers without truncation, i.e. alpha = max|g|: no
+    element is clipped and the largest element is reproduced exactly."""
+    rng = np.random.default_rng(21)
+    g = (rng.standard_t(2.5, 50_000) * 1e-3).astype(F32)
+    st = orc.stats(g)
+    for mode in (orc.UNIFORM, orc.NONUNIFORM):
+        p = orc.params(st, 8, mode, gamma=3.0, alpha_rule=orc.ALPHA_MAXABS)
+        assert p.alpha == st.max_abs and p.flags == 0
+        lv = p.levels_np()
+        assert lv[0] == -st.max_abs and lv[-1] == st.max_abs and np.all(np.diff(lv) > 0)
+        for x in g[:2000]:
+            assert orc.decision(p, float(x))[0] == float(x)          # T_alpha is the identity
+        j = int(np.argmax(np.abs(g)))
+        code = orc.code_from_bits(p, float(g[j]), 12345)
+        assert lv[code] == g[j]
+        # and it is a much coarser quantizer than the truncated one for a heavy tail
+        pt = orc.params(st, 8, mode, gamma=3.0)
+        assert p.alpha > 3 * pt.alpha
