@@ -210,6 +210,19 @@ tq_status tq_decompress_aggregate(const uint32_t* packed_dev, size_t words_strid
                                   float* out_dev, void* stream);
 
 /*
+ * Server side including the model update (Algorithm 1, last step: theta <- theta - eta * g_bar) with the
+ * optimiser of the paper's experiments (Section 5: momentum SGD with weight decay), fused into the
+ * aggregation so that g_bar never goes to memory:
+ *     g = g_bar_j (as tq_decompress_aggregate);  g += weight_decay * theta_j  (skipped when 0);
+ *     m_j = momentum * m_j + g  (when momentum_dev is given; g = m_j);  theta_j -= lr * g.
+ * fp32, every operation rounded once.  theta_dev [d] and momentum_dev [d] (may be NULL) are fp32 device
+ * arrays, 32-byte aligned, updated in place.  Other arguments and errors as tq_decompress_aggregate.
+ */
+tq_status tq_decompress_aggregate_apply(const uint32_t* packed_dev, size_t words_stride, uint32_t n_workers, uint64_t d,
+                                        const tq_params_t* params_host, const float* weights_host, float* theta_dev,
+                                        float* momentum_dev, float lr, float momentum, float weight_decay, void* stream);
+
+/*
  * The same round without a host round trip (the paper takes alpha and lambda_s as given inputs of
  * Algorithm 1; where they come from -- Section 4 -- can equally run on the device).
  *

@@ -111,6 +111,9 @@ def lib() -> C.CDLL:
         L.orc_compress.restype = i32
         L.orc_decompress_aggregate.argtypes = [C.c_void_p, u64, u32, u64, P(Params), C.c_void_p, C.c_void_p]
         L.orc_decompress_aggregate.restype = i32
+        L.orc_decompress_aggregate_apply.argtypes = [C.c_void_p, u64, u32, u64, P(Params), C.c_void_p, C.c_void_p,
+                                                     C.c_void_p, f32, f32, f32, C.c_void_p]
+        L.orc_decompress_aggregate_apply.restype = i32
         L.orc_sizeof_params.restype = u32; L.orc_sizeof_stats.restype = u32
         assert L.orc_sizeof_params() == C.sizeof(Params), "Params layout drifted from tq_oracle.c"
         assert L.orc_sizeof_stats() == C.sizeof(Stats), "Stats layout drifted from tq_oracle.c"
@@ -284,3 +287,22 @@ def decompress_aggregate(packed: np.ndarray, d: int, params_list: Sequence[Param
                                           None if w is None else w.ctypes.data, out.ctypes.data),
            "orc_decompress_aggregate")
     return out
+
+
+def decompress_aggregate_apply(packed: np.ndarray, d: int, params_list: Sequence[Params], theta: np.ndarray,
+                               momentum_buf: Optional[np.ndarray], lr: float, mu: float, wd: float,
+                               weights: Optional[Sequence[float]] = None):
+    """Aggregate and apply the model update in place on ``theta`` (and ``momentum_buf`` if given)."""
+    packed = np.ascontiguousarray(packed, dtype=np.uint32)
+    n = len(params_list)
+    arr = (Params * n)(*params_list)
+    assert theta.dtype == np.float32 and theta.flags.c_contiguous and theta.size == d
+    if momentum_buf is not None:
+        assert momentum_buf.dtype == np.float32 and momentum_buf.flags.c_contiguous and momentum_buf.size == d
+    scratch = np.empty(d, dtype=np.float32)
+    w = None if weights is None else _f32(weights)
+    _check(lib().orc_decompress_aggregate_apply(packed.ctypes.data, packed.shape[1], n, d, arr,
+                                                None if w is None else w.ctypes.data, theta.ctypes.data,
+                                                None if momentum_buf is None else momentum_buf.ctypes.data,
+                                                lr, mu, wd, scratch.ctypes.data), "orc_decompress_aggregate_apply")
+    return theta

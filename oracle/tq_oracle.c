@@ -56,6 +56,8 @@
  *       k = j/64 followed by 60 golden-section steps in the bracketing pair of cells; alpha iterates the
  *       boxed BiScaled equation as in R8 with k* recomputed at every step; s_alpha, s_beta are real
  *       numbers (the Appendix's formulas), so the levels come from the two-piece density by R7.
+ *   R18 the server's model update (Algorithm 1, last step) is the momentum SGD with weight decay of
+ *       Section 5: g += wd*theta; m = mu*m + g; theta -= lr*m; fp32, each operation rounded once.
  *   R13 aggregation: fp32 adds in worker order, then one IEEE division by N; with
  *       weights, each product w_i * v_i is rounded, then added, no division.
  */
@@ -612,6 +614,34 @@ int orc_decompress_aggregate(const uint32_t *packed, uint64_t stride_words, uint
             }
         }
         out[j] = weights ? acc : acc / (float)n_workers;
+    }
+    return ORC_OK;
+}
+
+/* Server side of Algorithm 1 including the model update (last step of the round), with the optimiser of
+ * the paper's experiments (Section 5: momentum SGD with weight decay).  R18: fp32, one rounding per
+ * operation: g = aggregate (R13); g += wd * theta (if wd != 0); m = mu * m + g (if a momentum buffer is
+ * given); theta -= lr * (m or g). */
+int orc_decompress_aggregate_apply(const uint32_t *packed, uint64_t stride_words, uint32_t n_workers,
+                                   uint64_t d, const orc_params_t *params, const float *weights,
+                                   float *theta, float *momentum_buf, float lr, float mu, float wd, float *scratch)
+{
+    int rc = orc_decompress_aggregate(packed, stride_words, n_workers, d, params, weights, scratch);
+    if (rc != ORC_OK) return rc;
+    for (uint64_t j = 0; j < d; ++j) {
+        float g = scratch[j];
+        if (wd != 0.0f) {
+            float decay = wd * theta[j];
+            g = g + decay;
+        }
+        if (momentum_buf) {
+            float carried = mu * momentum_buf[j];
+            float m = carried + g;
+            momentum_buf[j] = m;
+            g = m;
+        }
+        float step = lr * g;
+        theta[j] = theta[j] - step;
     }
     return ORC_OK;
 }

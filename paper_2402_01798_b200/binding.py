@@ -27,7 +27,7 @@ FLAG_ALPHA_CAPPED, FLAG_ALPHA_AT_GMIN, FLAG_GAMMA_FROM_MLE, FLAG_INVALID = 1, 2,
 
 EXPORTS = ("tq_packed_words", "tq_stats_workspace_bytes", "tq_stats", "tq_stats_static", "tq_params", "tq_params_batch", "tq_params_from_levels", "tq_params_device",
            "tq_compress_device_params", "tq_decompress_aggregate_device_params",
-           "tq_compress", "tq_decompress_aggregate", "tq_strerror", "tq_last_cuda_error", "tq_kernel_launches")
+           "tq_compress", "tq_decompress_aggregate", "tq_decompress_aggregate_apply", "tq_strerror", "tq_last_cuda_error", "tq_kernel_launches")
 
 
 class Stats(C.Structure):
@@ -87,6 +87,8 @@ def lib() -> C.CDLL:
         L.tq_compress_device_params.restype = C.c_int
         L.tq_decompress_aggregate_device_params.argtypes = [vp, sz, u32, u64, vp, u32, C.POINTER(f32), vp, vp]
         L.tq_decompress_aggregate_device_params.restype = C.c_int
+        L.tq_decompress_aggregate_apply.argtypes = [vp, sz, u32, u64, C.POINTER(Params), C.POINTER(f32), vp, vp, f32, f32, f32, vp]
+        L.tq_decompress_aggregate_apply.restype = C.c_int
         L.tq_strerror.argtypes = [C.c_int]; L.tq_strerror.restype = C.c_char_p
         L.tq_last_cuda_error.restype = C.c_int
         L.tq_kernel_launches.restype = u64
@@ -287,6 +289,19 @@ def tq_decompress_aggregate_device_params(packed: torch.Tensor, d: int, params_d
                                                        num_levels, w, out.data_ptr(), _stream(stream)),
            "tq_decompress_aggregate_device_params")
     return out
+
+
+def tq_decompress_aggregate_apply(packed: torch.Tensor, d: int, params, theta: torch.Tensor,
+                                  momentum_buf: Optional[torch.Tensor], lr: float, momentum: float = 0.0,
+                                  weight_decay: float = 0.0, weights: Optional[Sequence[float]] = None, stream=None):
+    """Aggregate the N packed rows and apply the SGD step in place on ``theta`` (and ``momentum_buf``)."""
+    n = packed.shape[0]
+    w = None if weights is None else (C.c_float * n)(*[float(x) for x in weights])
+    words_stride = packed.stride(0) if n > 1 else packed.shape[1]
+    _check(lib().tq_decompress_aggregate_apply(packed.data_ptr(), words_stride, n, d, _params_array(params), w,
+                                               theta.data_ptr(), None if momentum_buf is None else momentum_buf.data_ptr(),
+                                               lr, momentum, weight_decay, _stream(stream)), "tq_decompress_aggregate_apply")
+    return theta
 
 
 def tq_kernel_launches() -> int:

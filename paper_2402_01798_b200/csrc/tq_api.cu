@@ -182,6 +182,27 @@ tq_status tq_decompress_aggregate_device_params(const uint32_t* packed_dev, size
     return TQ_OK;
 }
 
+tq_status tq_decompress_aggregate_apply(const uint32_t* packed_dev, size_t words_stride, uint32_t n_workers, uint64_t d,
+                                        const tq_params_t* params_host, const float* weights_host, float* theta_dev,
+                                        float* momentum_dev, float lr, float momentum, float weight_decay, void* stream) {
+    if (n_workers == 0 || n_workers > TQ_MAX_WORKERS || d > (1ull << 40)) return TQ_ERR_INVALID_ARG;
+    uint32_t bits = 0;
+    if (tq_status s = check_params(params_host, n_workers, &bits)) return s;
+    const size_t need = tq_packed_words(d, bits);
+    if (d && (!packed_dev || !theta_dev)) return TQ_ERR_INVALID_ARG;
+    if (!(lr == lr) || !(momentum == momentum) || !(weight_decay == weight_decay)) return TQ_ERR_INVALID_ARG;
+    if (!aligned(packed_dev, 16) || words_stride % 4 != 0 || !aligned(theta_dev, 32) || !aligned(momentum_dev, 32)) return TQ_ERR_ALIGNMENT;
+    if (words_stride < need) return TQ_ERR_BUFFER_TOO_SMALL;
+    if (d == 0) return TQ_OK;
+    tq::DecompressCall c{packed_dev, words_stride, need, n_workers, d, params_host, nullptr, weights_host, bits, nullptr,
+                         static_cast<cudaStream_t>(stream)};
+    c.theta = theta_dev; c.momentum_buf = momentum_dev; c.lr = lr; c.mu = momentum; c.wd = weight_decay;
+    const cudaError_t e = tq::launch_decompress(c);
+    if (e != cudaSuccess) return cuda_failed(e);
+    g_launches += 1;
+    return TQ_OK;
+}
+
 const char* tq_strerror(tq_status s) {
     switch (s) {
         case TQ_OK: return "ok";

@@ -18,6 +18,13 @@ struct DecompressArgs {
     float table[TQ_MAX_WORKERS][TQ_MAX_LEVELS];   // levels, already multiplied by w_i when weights are given
 };
 // Device-resident parameters: the codebooks are read from params_dev by each block; weights by value.
+// Optional fused model update (Algorithm 1, last step, with the momentum SGD + weight decay of the
+// paper's experiments): theta and the momentum buffer are read and written instead of `out`.
+struct ApplyArgs {
+    float* theta;          // nullptr: plain aggregation into `out`
+    float* momentum_buf;   // may be nullptr (no momentum)
+    float lr, mu, wd;
+};
 struct DeviceTables {
     const tq_params_t* params_dev;    // nullptr: use DecompressArgs
     int use_weights;
@@ -119,11 +126,11 @@ __device__ __forceinline__ void add_unit(f32x2* acc, uint32_t f, const char* tab
 #define TQ_DECOMPRESS_MIN_BLOCKS 4
 #endif
 
-template <int BITS>
+template <int BITS, bool APPLY>
 __global__ void __launch_bounds__(kThreads, TQ_DECOMPRESS_MIN_BLOCKS)
 decompress_kernel(const uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_valid, uint32_t n,
                   uint64_t d, const __grid_constant__ DecompressArgs args, const __grid_constant__ DeviceTables dt,
-                  float scale, int divide,
+                  float scale, int divide, const __grid_constant__ ApplyArgs ap,
                   float* __restrict__ out) {
     constexpr int E = Unit<BITS>::kElems, U = Unit<BITS>::kUnits;
 
@@ -198,7 +205,37 @@ decompress_kernel(const uint32_t* __restrict__ packed, uint64_t words_stride, ui
         }
         const uint64_t u = u0 + static_cast<uint64_t>(k) * kThreads;
         const uint64_t j0 = u * E;
-        if (j0 + E <= d) {
+        const bool whole = j0 + E <= d;
+        if constexpr (APPLY) {
+            // g += wd * theta; m = mu * m + g; theta -= lr * (m or g): fp32, one rounding per operation
+#pragma unroll
+            for (int v = 0; v < E / 8; ++v) {
+                float th[8], mo[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const uint64_t j = j0 + 8 * v + e;
+                    th[e] = (whole || j < d) ? ap.theta[j] : 0.0f;
+                    mo[e] = (ap.momentum_buf && (whole || j < d)) ? ap.momentum_buf[j] : 0.0f;
+                }
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    float gj = o[8 * v + e];
+                    if (ap.wd != 0.0f) gj = __fadd_rn(gj, __fmul_rn(ap.wd, th[e]));
+                    if (ap.momentum_buf) { mo[e] = __fadd_rn(__fmul_rn(ap.mu, mo[e]), gj); gj = mo[e]; }
+                    th[e] = __fsub_rn(th[e], __fmul_rn(ap.lr, gj));
+                }
+                if (whole) {
+                    stg256(ap.theta + j0 + 8 * v, th);
+                    if (ap.momentum_buf) stg256(ap.momentum_buf + j0 + 8 * v, mo);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const uint64_t j = j0 + 8 * v + e;
+                        if (j < d) { ap.theta[j] = th[e]; if (ap.momentum_buf) ap.momentum_buf[j] = mo[e]; }
+                    }
+                }
+            }
+        } else if (whole) {
 #pragma unroll
             for (int v = 0; v < E / 8; ++v) {
                 const float o8[8] = {o[8 * v], o[8 * v + 1], o[8 * v + 2], o[8 * v + 3],
@@ -220,8 +257,13 @@ static cudaError_t launch(const DecompressCall& c, const DecompressArgs& args, c
     const uint64_t blocks = (n_units + per_block - 1) / per_block;
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7FFFFFFFull) return cudaErrorInvalidConfiguration;
-    decompress_kernel<BITS><<<static_cast<unsigned>(blocks), kThreads, 0, c.stream>>>(
-        c.packed, c.words_stride, c.words_valid, c.n_workers, c.d, args, dt, scale, divide, c.out);
+    const ApplyArgs ap{c.theta, c.momentum_buf, c.lr, c.mu, c.wd};
+    if (c.theta)
+        decompress_kernel<BITS, true><<<static_cast<unsigned>(blocks), kThreads, 0, c.stream>>>(
+            c.packed, c.words_stride, c.words_valid, c.n_workers, c.d, args, dt, scale, divide, ap, c.out);
+    else
+        decompress_kernel<BITS, false><<<static_cast<unsigned>(blocks), kThreads, 0, c.stream>>>(
+            c.packed, c.words_stride, c.words_valid, c.n_workers, c.d, args, dt, scale, divide, ap, c.out);
     return cudaGetLastError();
 }
 

@@ -24,6 +24,7 @@ struct DecompressCall {
     const tq_params_t* params_dev;   // device array (then bits comes from the caller)
     const float* weights; uint32_t bits;
     float* out; cudaStream_t stream;
+    float* theta = nullptr; float* momentum_buf = nullptr; float lr = 0.0f, mu = 0.0f, wd = 0.0f;   // fused model update
 };
 cudaError_t launch_decompress(const DecompressCall& c);
 

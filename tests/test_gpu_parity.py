@@ -460,3 +460,34 @@ def test_device_params_marks_bad_statistics_and_fallback_codebooks(tq, orc):
     pk = tq.tq_compress_device_params(g2, raw, 8, tq.NONUNIFORM, seed=9, d=d).cpu().numpy().view(np.uint32)
     for i in range(n):
         assert np.array_equal(pk[i], orc.compress(host_f32(orc, g2[i, :d]), to_oracle_params(orc, p), 9, i))
+
+
+@pytest.mark.parametrize("bits,n,mu,wd", [(4, 16, 0.9, 5e-4), (3, 4, 0.9, 0.0), (2, 8, 0.0, 1e-3), (4, 3, 0.0, 0.0), (1, 2, 0.5, 5e-4)])
+def test_fused_model_update_matches_oracle(tq, orc, bits, n, mu, wd):
+    """tq_decompress_aggregate_apply: aggregation fused with the momentum-SGD step, two rounds in a row,
+    theta and the momentum buffer bit-exact against the oracle (ragged d, canaries past the end)."""
+    L = 1 << bits
+    rng = np.random.default_rng(bits * 31 + n)
+    for d in (33, 100_003):
+        ps = []
+        for i in range(n):
+            a = 0.01 * (1 + 0.3 * i)
+            mags = np.geomspace(a / 50, a, L // 2).astype(F32) if L > 2 else np.array([a], dtype=F32)
+            ps.append(tq.tq_params_from_levels([float(x) for x in np.concatenate([-mags[::-1], mags])]))
+        ops = [to_oracle_params(orc, p) for p in ps]
+        theta_h = rng.normal(0, 0.1, d).astype(F32)
+        buf_h = np.zeros(d, dtype=F32) if mu != 0.0 else None
+        theta = torch.full((d + 16,), 5.0, dtype=torch.float32, device="cuda"); theta[:d] = torch.from_numpy(theta_h)
+        buf = None
+        if mu != 0.0:
+            buf = torch.full((d + 16,), -3.0, dtype=torch.float32, device="cuda"); buf[:d] = 0.0
+        for rnd in range(2):
+            codes = rng.integers(0, L, (n, d), dtype=np.uint8)
+            packed_h = np.stack([orc.pack(codes[i], bits) for i in range(n)])
+            packed = torch.from_numpy(packed_h.view(np.int32)).cuda()
+            tq.tq_decompress_aggregate_apply(packed, d, ps, theta, buf, 0.01, mu, wd)
+            orc.decompress_aggregate_apply(packed_h, d, ops, theta_h, buf_h, 0.01, mu, wd)
+            assert np.array_equal(theta[:d].cpu().numpy(), theta_h)
+            assert bool((theta[d:] == 5.0).all())
+            if buf is not None:
+                assert np.array_equal(buf[:d].cpu().numpy(), buf_h) and bool((buf[d:] == -3.0).all())

@@ -37,6 +37,8 @@ MUTATIONS = [
     ("biscaled density split", "double denom = 2.0 * c2 * (1.0 - k) * alpha + 2.0 * c1 * k * alpha;", "double denom = 2.0 * c2 * k * alpha + 2.0 * c1 * (1.0 - k) * alpha;", "test_oracle_biscaled.py"),
     ("biscaled level offset", "double c = (double)k - 0.5 * (double)s;", "double c = (double)k - 0.5 * (double)(s + 1);", "test_oracle_biscaled.py"),
     ("biscaled inner mass", "double p1 = orc_model_QU(m, beta) / (2.0 * beta);", "double p1 = orc_model_QU(m, beta) / beta;", "test_oracle_biscaled.py"),
+    ("update sign", "theta[j] = theta[j] - step;", "theta[j] = theta[j] + step;", "test_oracle_pack_aggregate.py"),
+    ("momentum order", "float m = carried + g;", "float m = carried + lr * g;", "test_oracle_pack_aggregate.py"),
     ("cube root dropped", "double cb = cbrt((1.0 - 2.0 * m->rho) / (2.0 * m->g_min));\n    if (x <= m->g_min) return cb * x;", "double cb = (1.0 - 2.0 * m->rho) / (2.0 * m->g_min);\n    if (x <= m->g_min) return cb * x;", "test_oracle_params.py"),
 ]
 

@@ -143,3 +143,43 @@ def test_round_trip_mean_is_close_to_clipped_mean(orc):
     widths = np.diff(p.levels_np()).max()
     assert np.abs(out - clip).max() < 5 * widths / 2 / np.sqrt(n)
     assert abs(np.mean(out - clip)) < 4 * widths / 2 / np.sqrt(n * d)
+
+
+def _sgd_reference(theta, buf, g, lr, mu, wd):
+    """fp32 momentum SGD with weight decay, one NumPy fp32 operation per step (independent restatement)."""
+    g = g.astype(F32)
+    if wd != 0.0:
+        g = (g + (F32(wd) * theta).astype(F32)).astype(F32)
+    if buf is not None:
+        buf[:] = ((F32(mu) * buf).astype(F32) + g).astype(F32)
+        g = buf
+    theta[:] = (theta - (F32(lr) * g).astype(F32)).astype(F32)
+
+
+@pytest.mark.parametrize("mu,wd", [(0.9, 5e-4), (0.0, 0.0), (0.9, 0.0), (0.0, 1e-2)])
+def test_fused_model_update_is_momentum_sgd(orc, mu, wd):
+    """Algorithm 1's last step with the optimiser of Section 5 (momentum SGD, lr 0.01, momentum 0.9,
+    weight decay 5e-4): three rounds in a row against a step-by-step fp32 restatement and against
+    torch.optim.SGD (which may fuse a multiply-add: compared to 1e-6)."""
+    import torch
+    rng = np.random.default_rng(5)
+    n, d, bits = 4, 1237, 3
+    ps = _tables(orc, n, 8, orc.NONUNIFORM)
+    theta = rng.normal(0, 0.1, d).astype(F32)
+    use_buf = mu != 0.0
+    buf = np.zeros(d, dtype=F32) if use_buf else None
+    th_ref, buf_ref = theta.copy(), (buf.copy() if use_buf else None)
+    pt = torch.nn.Parameter(torch.from_numpy(theta.copy()))
+    opt = torch.optim.SGD([pt], lr=0.01, momentum=mu, weight_decay=wd)
+    for rnd in range(3):
+        codes = rng.integers(0, 8, (n, d), dtype=np.uint8)
+        packed = np.stack([orc.pack(codes[i], bits) for i in range(n)])
+        gbar = orc.decompress_aggregate(packed, d, ps)
+        orc.decompress_aggregate_apply(packed, d, ps, theta, buf, 0.01, mu, wd)
+        _sgd_reference(th_ref, buf_ref, gbar, 0.01, mu, wd)
+        assert np.array_equal(theta, th_ref)
+        if use_buf:
+            assert np.array_equal(buf, buf_ref)
+        pt.grad = torch.from_numpy(gbar.copy())
+        opt.step()
+        assert np.allclose(theta, pt.detach().numpy(), rtol=1e-6, atol=1e-9)
