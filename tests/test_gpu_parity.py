@@ -491,3 +491,35 @@ def test_fused_model_update_matches_oracle(tq, orc, bits, n, mu, wd):
             assert bool((theta[d:] == 5.0).all())
             if buf is not None:
                 assert np.array_equal(buf[:d].cpu().numpy(), buf_h) and bool((buf[d:] == -3.0).all())
+
+
+def test_layer_groups_are_quantized_independently(tq, orc):
+    """Section 5: convolutional and fully-connected gradients have different distributions and are
+    quantized independently.  With row strides in the ABI a layer group is a column range of the
+    [N, d] gradient block: one statistics / compress / decompress call per group on a 32-byte aligned
+    sub-range, each group with its own alpha and codebook, element indices counted within the group."""
+    n, d_conv, d_fc = 4, 60_000, 140_008
+    d = d_conv + d_fc
+    g = torch.zeros((n, d), dtype=torch.float32, device="cuda")
+    from paper_2402_01798_b200 import inputs
+    for i in range(n):
+        inputs.powerlaw_gradient(d_conv, 4.0, 5e-3, 900 + i, "cuda", out=g[i, :d_conv])       # light tail, large scale
+        inputs.powerlaw_gradient(d_fc, 2.5, 2e-4, 950 + i, "cuda", out=g[i, d_conv:])        # heavy tail, small scale
+    out = torch.empty(d, dtype=torch.float32, device="cuda")
+    alphas = []
+    for lo, hi, gamma, L, mode in ((0, d_conv, 4.0, 8, tq.UNIFORM), (d_conv, d, 2.5, 8, tq.NONUNIFORM)):
+        view = g[:, lo:hi]
+        st = tq.stats_to_host(tq.tq_stats(view))
+        ps = [tq.tq_params(s, L, mode, gamma) for s in st]
+        alphas.append(ps[0].alpha)
+        packed = tq.tq_compress(view, ps, seed=17)
+        tq.tq_decompress_aggregate(packed, hi - lo, ps, out=out[lo:hi])
+        ops = [to_oracle_params(orc, p) for p in ps]
+        got = packed.cpu().numpy().view(np.uint32)
+        for i in range(n):
+            x = host_f32(orc, g[i, lo:hi])
+            o = orc.stats(x, g_min=st[i].g_min)
+            assert o.n_tail == st[i].n_tail and math.isclose(o.sum_abs, st[i].sum_abs, rel_tol=TOL_SUM)
+            assert np.array_equal(got[i], orc.compress(x, ops[i], 17, i))
+        assert np.array_equal(out[lo:hi].cpu().numpy(), orc.decompress_aggregate(got, hi - lo, ops))
+    assert max(alphas) > 5 * min(alphas)      # the groups really get different thresholds
