@@ -183,3 +183,16 @@ def test_fused_model_update_is_momentum_sgd(orc, mu, wd):
         pt.grad = torch.from_numpy(gbar.copy())
         opt.step()
         assert np.allclose(theta, pt.detach().numpy(), rtol=1e-6, atol=1e-9)
+
+
+def test_oracle_outputs_match_the_stored_checksums():
+    """tests/golden/oracle_small_case.txt is written by tests/golden/make_oracle_golden.py from the oracle
+    alone; a mismatch means the oracle's arithmetic (or its inputs) changed."""
+    import importlib.util
+    import os
+    here = os.path.join(os.path.dirname(__file__), "golden")
+    spec = importlib.util.spec_from_file_location("make_oracle_golden", os.path.join(here, "make_oracle_golden.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    stored = open(os.path.join(here, "oracle_small_case.txt")).read().splitlines()
+    assert mod.lines() == stored
