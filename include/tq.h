@@ -254,6 +254,15 @@ const char* tq_strerror(tq_status status);
 int tq_last_cuda_error(void);   /* cudaError_t of the last failed runtime call on this thread, else 0 */
 uint64_t tq_kernel_launches(void); /* kernels launched by this library in this process so far */
 
+/* Bounded waits.  The large-input decompression kernel stages packed bytes through asynchronous bulk
+ * copies and waits for them on shared-memory barriers; every such wait gives up after a fixed number
+ * of polls.  A block whose wait ran out stores nothing for its tile and counts itself here.
+ * *count_host receives the number of such give-ups on the current device since the library was loaded
+ * (0 in a healthy run: a non-zero value means the outputs of the affected launch are incomplete).
+ * Synchronises the device.  Returns TQ_ERR_INVALID_ARG for a null pointer, TQ_ERR_CUDA if the read fails.
+ * (The paper has no counterpart; this is a health check of the implementation.) */
+tq_status tq_wait_expired_count(uint32_t* count_host);
+
 #ifdef __cplusplus
 }
 #endif

@@ -27,7 +27,7 @@ FLAG_ALPHA_CAPPED, FLAG_ALPHA_AT_GMIN, FLAG_GAMMA_FROM_MLE, FLAG_INVALID = 1, 2,
 
 EXPORTS = ("tq_packed_words", "tq_stats_workspace_bytes", "tq_stats", "tq_stats_static", "tq_params", "tq_params_batch", "tq_params_from_levels", "tq_params_device",
            "tq_compress_device_params", "tq_decompress_aggregate_device_params",
-           "tq_compress", "tq_decompress_aggregate", "tq_decompress_aggregate_apply", "tq_strerror", "tq_last_cuda_error", "tq_kernel_launches")
+           "tq_compress", "tq_decompress_aggregate", "tq_decompress_aggregate_apply", "tq_strerror", "tq_last_cuda_error", "tq_kernel_launches", "tq_wait_expired_count")
 
 
 class Stats(C.Structure):
@@ -92,6 +92,7 @@ def lib() -> C.CDLL:
         L.tq_strerror.argtypes = [C.c_int]; L.tq_strerror.restype = C.c_char_p
         L.tq_last_cuda_error.restype = C.c_int
         L.tq_kernel_launches.restype = u64
+        L.tq_wait_expired_count.argtypes = [C.POINTER(u32)]; L.tq_wait_expired_count.restype = C.c_int
         _lib = L
     return _lib
 
@@ -306,3 +307,10 @@ def tq_decompress_aggregate_apply(packed: torch.Tensor, d: int, params, theta: t
 
 def tq_kernel_launches() -> int:
     return int(lib().tq_kernel_launches())
+
+
+def tq_wait_expired_count() -> int:
+    """Give-ups of bounded barrier waits inside the library's kernels on the current device (0 when healthy)."""
+    n = C.c_uint32(0)
+    _check(lib().tq_wait_expired_count(C.byref(n)), "tq_wait_expired_count")
+    return int(n.value)

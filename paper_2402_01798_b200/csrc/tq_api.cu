@@ -220,4 +220,13 @@ const char* tq_strerror(tq_status s) {
 int tq_last_cuda_error(void) { return g_last_cuda_error; }
 uint64_t tq_kernel_launches(void) { return g_launches.load(); }
 
+tq_status tq_wait_expired_count(uint32_t* count_host) {
+    if (!count_host) return TQ_ERR_INVALID_ARG;
+    unsigned int n = 0;
+    const cudaError_t e = tq::read_wait_expired(&n);
+    if (e != cudaSuccess) return cuda_failed(e);
+    *count_host = n;
+    return TQ_OK;
+}
+
 }  // extern "C"

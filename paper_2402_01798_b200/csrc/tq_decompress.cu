@@ -122,82 +122,15 @@ __device__ __forceinline__ void add_unit(f32x2* acc, uint32_t f, const char* tab
     }
 }
 
-// Blocks of 128 threads, eight resident per SM: the same 32 warps per SM as four blocks of 256, but
-// a block that reaches its tail or its barrier leaves fewer lanes idle (measured 2-3 % faster).
-// The fused update holds theta and the momentum buffer as well and gets two blocks fewer, which
-// keeps it free of spills.
 constexpr int kDecThreads = 128;
-#ifndef TQ_DECOMPRESS_MIN_BLOCKS
-#define TQ_DECOMPRESS_MIN_BLOCKS 8
-#endif
 
+// Turns the accumulated sums of a thread's units into outputs: the division by N (w_i = 1/N; for N a
+// power of two the product with 2^-k is the same value), then either the store of the aggregate or
+// the fused model update.  Unit k of the thread is unit u0 + k * kDecThreads of the row.
 template <int BITS, bool APPLY>
-__global__ void __launch_bounds__(kDecThreads, APPLY ? TQ_DECOMPRESS_MIN_BLOCKS - 2 : TQ_DECOMPRESS_MIN_BLOCKS)
-decompress_kernel(const uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_valid, uint32_t n,
-                  uint64_t d, const __grid_constant__ DecompressArgs args, const __grid_constant__ DeviceTables dt,
-                  float scale, int divide, const __grid_constant__ ApplyArgs ap,
-                  float* __restrict__ out) {
+__device__ __forceinline__ void finish_units(f32x2 (&acc)[Unit<BITS>::kUnits][Unit<BITS>::kElems / 2], uint64_t u0, uint64_t d,
+                                             float scale, int divide, const ApplyArgs& ap, float* __restrict__ out) {
     constexpr int E = Unit<BITS>::kElems, U = Unit<BITS>::kUnits;
-
-    // Each worker's codebook starts on a 256-byte boundary of shared memory, so a table offset
-    // (code * 4 < 64) can be merged into the worker's base offset by the same byte-permute that
-    // extracts it.  Bank = code: the lookups of one instruction never conflict.
-    __shared__ __align__(256) float s_tab[TQ_MAX_WORKERS * kTabStride];
-    for (uint32_t t = threadIdx.x; t < n * TQ_MAX_LEVELS; t += kDecThreads) {
-        const uint32_t i = t / TQ_MAX_LEVELS, k = t % TQ_MAX_LEVELS;
-        float v;
-        if (dt.params_dev) {     // same rounded product w_i * l as the host forms for the by-value table
-            const float l = dt.params_dev[i].levels[k];
-            v = dt.use_weights ? __fmul_rn(dt.weights[i], l) : l;
-        } else {
-            v = args.table[i][k];
-        }
-        s_tab[i * kTabStride + k] = v;
-    }
-    __syncthreads();
-    const char* tab_bytes = reinterpret_cast<const char*>(s_tab);
-
-    const uint64_t n_units = (d + E - 1) / E;
-    const uint64_t u0 = static_cast<uint64_t>(blockIdx.x) * (kDecThreads * U) + threadIdx.x;   // unit k of this thread: u0 + k * kDecThreads
-    if (u0 >= n_units) return;
-
-    f32x2 acc[U][E / 2];          // fp32 accumulators, two per 64-bit register pair
-#pragma unroll
-    for (int k = 0; k < U; ++k)
-#pragma unroll
-        for (int e = 0; e < E / 2; ++e) acc[k][e] = both(0.0f);
-
-    // interior: all U units exist and all their words lie inside the row
-    const uint64_t u_last = u0 + static_cast<uint64_t>(U - 1) * kDecThreads;
-    const bool interior = u_last < n_units && last_word_of<BITS>(u_last) < words_valid;
-
-    uint32_t i = 0;
-    if (interior) {
-        for (; i + 4 <= n; i += 4) {          // four workers at a time: 4 * U independent fields in flight
-            uint32_t f[4][U];
-#pragma unroll
-            for (int b = 0; b < 4; ++b)
-#pragma unroll
-                for (int k = 0; k < U; ++k)
-                    f[b][k] = load_field<BITS>(packed + static_cast<uint64_t>(i + b) * words_stride, u0 + k * kDecThreads);
-#pragma unroll
-            for (int b = 0; b < 4; ++b)
-#pragma unroll
-                for (int k = 0; k < U; ++k)
-                    add_unit<BITS>(acc[k], f[b][k], tab_bytes + b * (kTabStride * 4), i * (kTabStride * 4));
-        }
-    }
-    for (; i < n; ++i) {                       // remaining workers, or every worker of an edge thread
-        uint32_t f[U];
-#pragma unroll
-        for (int k = 0; k < U; ++k)
-            f[k] = load_field_guarded<BITS>(packed + static_cast<uint64_t>(i) * words_stride,
-                                            u0 + static_cast<uint64_t>(k) * kDecThreads, words_valid);
-#pragma unroll
-        for (int k = 0; k < U; ++k) add_unit<BITS>(acc[k], f[k], tab_bytes, i * (kTabStride * 4));
-    }
-
-    // w_i = 1/N: one division by N (for N a power of two the product with 2^-k is the same value)
 #pragma unroll
     for (int k = 0; k < U; ++k) {
         float o[E];
@@ -255,6 +188,255 @@ decompress_kernel(const uint32_t* __restrict__ packed, uint64_t words_stride, ui
     }
 }
 
+// Copies the N codebooks (already multiplied by w_i when weights are given) into shared memory.
+__device__ __forceinline__ void fill_tables(float* s_tab, uint32_t n, const DecompressArgs& args, const DeviceTables& dt) {
+    for (uint32_t t = threadIdx.x; t < n * TQ_MAX_LEVELS; t += kDecThreads) {
+        const uint32_t i = t / TQ_MAX_LEVELS, k = t % TQ_MAX_LEVELS;
+        float v;
+        if (dt.params_dev) {     // same rounded product w_i * l as the host forms for the by-value table
+            const float l = dt.params_dev[i].levels[k];
+            v = dt.use_weights ? __fmul_rn(dt.weights[i], l) : l;
+        } else {
+            v = args.table[i][k];
+        }
+        s_tab[i * kTabStride + k] = v;
+    }
+}
+
+// Blocks of 128 threads, eight resident per SM: the same 32 warps per SM as four blocks of 256, but
+// a block that reaches its tail or its barrier leaves fewer lanes idle (measured 2-3 % faster).
+// The fused update holds theta and the momentum buffer as well and gets two blocks fewer, which
+// keeps it free of spills.
+#ifndef TQ_DECOMPRESS_MIN_BLOCKS
+#define TQ_DECOMPRESS_MIN_BLOCKS 8
+#endif
+
+template <int BITS, bool APPLY>
+__global__ void __launch_bounds__(kDecThreads, APPLY ? TQ_DECOMPRESS_MIN_BLOCKS - 2 : TQ_DECOMPRESS_MIN_BLOCKS)
+decompress_kernel(const uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_valid, uint32_t n,
+                  uint64_t d, const __grid_constant__ DecompressArgs args, const __grid_constant__ DeviceTables dt,
+                  float scale, int divide, const __grid_constant__ ApplyArgs ap,
+                  float* __restrict__ out) {
+    constexpr int E = Unit<BITS>::kElems, U = Unit<BITS>::kUnits;
+
+    // Each worker's codebook starts on a 256-byte boundary of shared memory, so a table offset
+    // (code * 4 < 64) can be merged into the worker's base offset by the same byte-permute that
+    // extracts it.  Bank = code: the lookups of one instruction never conflict.
+    __shared__ __align__(256) float s_tab[TQ_MAX_WORKERS * kTabStride];
+    fill_tables(s_tab, n, args, dt);
+    __syncthreads();
+    const char* tab_bytes = reinterpret_cast<const char*>(s_tab);
+
+    const uint64_t n_units = (d + E - 1) / E;
+    const uint64_t u0 = static_cast<uint64_t>(blockIdx.x) * (kDecThreads * U) + threadIdx.x;   // unit k of this thread: u0 + k * kDecThreads
+    if (u0 >= n_units) return;
+
+    f32x2 acc[U][E / 2];          // fp32 accumulators, two per 64-bit register pair
+#pragma unroll
+    for (int k = 0; k < U; ++k)
+#pragma unroll
+        for (int e = 0; e < E / 2; ++e) acc[k][e] = both(0.0f);
+
+    // interior: all U units exist and all their words lie inside the row
+    const uint64_t u_last = u0 + static_cast<uint64_t>(U - 1) * kDecThreads;
+    const bool interior = u_last < n_units && last_word_of<BITS>(u_last) < words_valid;
+
+    uint32_t i = 0;
+    if (interior) {
+        for (; i + 4 <= n; i += 4) {          // four workers at a time: 4 * U independent fields in flight
+            uint32_t f[4][U];
+#pragma unroll
+            for (int b = 0; b < 4; ++b)
+#pragma unroll
+                for (int k = 0; k < U; ++k)
+                    f[b][k] = load_field<BITS>(packed + static_cast<uint64_t>(i + b) * words_stride, u0 + k * kDecThreads);
+#pragma unroll
+            for (int b = 0; b < 4; ++b)
+#pragma unroll
+                for (int k = 0; k < U; ++k)
+                    add_unit<BITS>(acc[k], f[b][k], tab_bytes + b * (kTabStride * 4), i * (kTabStride * 4));
+        }
+    }
+    for (; i < n; ++i) {                       // remaining workers, or every worker of an edge thread
+        uint32_t f[U];
+#pragma unroll
+        for (int k = 0; k < U; ++k)
+            f[k] = load_field_guarded<BITS>(packed + static_cast<uint64_t>(i) * words_stride,
+                                            u0 + static_cast<uint64_t>(k) * kDecThreads, words_valid);
+#pragma unroll
+        for (int k = 0; k < U; ++k) add_unit<BITS>(acc[k], f[k], tab_bytes, i * (kTabStride * 4));
+    }
+
+    finish_units<BITS, APPLY>(acc, u0, d, scale, divide, ap, out);
+}
+
+
+// ---------------------------------------------------------------------------------------------
+// Bulk-copy variant for large inputs.  One block decodes one tile of kDecThreads * 32 outputs.  The
+// packed bytes of the tile, kGroup workers at a time, are brought into a ring of shared-memory stages
+// by asynchronous bulk copies (one per worker row, completion counted on an mbarrier), so the next
+// workers' bytes are in flight while the current ones are looked up, and no registers are tied up by
+// loads in flight.  A worker's bytes of one tile are contiguous in its row, start on a 16-byte
+// boundary and are a multiple of 16 bytes long (rows are padded to 16 bytes), as a bulk copy needs.
+// Every wait on a barrier is bounded; a wait that runs out makes the block count itself in
+// g_wait_expired, wait (bounded again) for its copies still in flight and return without storing.
+constexpr int kGroup = 4;                     // workers per stage
+#ifndef TQ_DECOMPRESS_STAGES
+#define TQ_DECOMPRESS_STAGES 2
+#endif
+constexpr uint32_t kWaitLimit = 1u << 22;     // polls of one barrier before giving up
+
+__device__ unsigned int g_wait_expired = 0;   // blocks (or threads) whose bounded wait ran out, since load
+
+template <int BITS>
+struct Tile {
+    static constexpr int kUnitBytes = BITS == 3 ? 3 : 4;
+    static constexpr int kUnits = kDecThreads * Unit<BITS>::kUnits;     // units per tile (a multiple of 4)
+    static constexpr int kSegBytes = kUnits * kUnitBytes;               // one worker's bytes per tile (a multiple of 16)
+};
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// global -> this block's shared memory, `bytes` a multiple of 16, both addresses 16-byte aligned
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t it = 0; it < kWaitLimit; ++it) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+// The field of local unit ul of a tile segment in shared memory (same cut as load_field; the tile's
+// first unit is a multiple of 4, so the byte phase of a 3-bit unit is that of its local index).
+template <int BITS>
+__device__ __forceinline__ uint32_t stage_field(const uint32_t* seg, uint32_t ul) {
+    if constexpr (BITS != 3) return seg[ul];
+    else {
+        const uint32_t wi = (3u * ul) >> 2, sh = (ul * 24u) & 31u;
+        return __funnelshift_r(seg[wi], seg[wi + 1], sh);
+    }
+}
+
+template <int BITS, bool APPLY>
+__global__ void __launch_bounds__(kDecThreads, APPLY ? TQ_DECOMPRESS_MIN_BLOCKS - 2 : TQ_DECOMPRESS_MIN_BLOCKS)
+decompress_bulk_kernel(const uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_valid, uint32_t n,
+                       uint64_t d, const __grid_constant__ DecompressArgs args, const __grid_constant__ DeviceTables dt,
+                       float scale, int divide, const __grid_constant__ ApplyArgs ap, float* __restrict__ out) {
+    constexpr int E = Unit<BITS>::kElems, U = Unit<BITS>::kUnits, S = TQ_DECOMPRESS_STAGES;
+    constexpr uint32_t kSeg = Tile<BITS>::kSegBytes;
+
+    // [codebooks: n * 256 B][S stages of kGroup segments][16 B that a 3-bit field's second word may touch][S barriers]
+    extern __shared__ __align__(1024) unsigned char smem[];
+    float* s_tab = reinterpret_cast<float*>(smem);
+    unsigned char* s_stage = smem + static_cast<size_t>(n) * (kTabStride * 4);
+    const uint32_t stage0 = smem_addr(s_stage);
+    const uint32_t bar0 = stage0 + S * kGroup * kSeg + 16;
+
+    const uint64_t tile = blockIdx.x;
+    const uint64_t tile_off = tile * kSeg;                                   // byte offset of the tile in every row
+    const uint64_t row_bytes = words_valid * 4;
+    const uint32_t seg_bytes = static_cast<uint32_t>(row_bytes - tile_off < kSeg ? row_bytes - tile_off : kSeg);
+    const uint32_t n_steps = (n + kGroup - 1) / kGroup;
+    const char* src0 = reinterpret_cast<const char*>(packed) + tile_off;
+
+    // step q = workers q*kGroup .. ; its bytes go to stage q % S
+    auto issue = [&](uint32_t q) {
+        const uint32_t st = q % S, i0 = q * kGroup;
+        const uint32_t cnt = n - i0 < kGroup ? n - i0 : kGroup;
+        const uint32_t bar = bar0 + 8 * st;
+        mbar_expect_tx(bar, cnt * seg_bytes);
+        for (uint32_t b = 0; b < cnt; ++b)
+            bulk_load(stage0 + (st * kGroup + b) * kSeg, src0 + static_cast<uint64_t>(i0 + b) * words_stride * 4, seg_bytes, bar);
+    };
+
+    if (threadIdx.x == 0) {
+        for (int st = 0; st < S; ++st) mbar_init(bar0 + 8 * st, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        for (uint32_t q = 0; q < S && q < n_steps; ++q) issue(q);
+    }
+    fill_tables(s_tab, n, args, dt);
+    __syncthreads();          // barriers initialised and codebooks in place for every thread
+    const char* tab_bytes = reinterpret_cast<const char*>(s_tab);
+
+    f32x2 acc[U][E / 2];
+#pragma unroll
+    for (int k = 0; k < U; ++k)
+#pragma unroll
+        for (int e = 0; e < E / 2; ++e) acc[k][e] = both(0.0f);
+
+    uint32_t q = 0;
+    bool expired = false;
+    for (; q < n_steps; ++q) {
+        const uint32_t st = q % S, i0 = q * kGroup;
+        const uint32_t cnt = n - i0 < kGroup ? n - i0 : kGroup;
+        const bool ok = mbar_wait(bar0 + 8 * st, (q / S) & 1u);
+        uint32_t f[kGroup][U];
+        const uint32_t* seg = reinterpret_cast<const uint32_t*>(s_stage + static_cast<size_t>(st) * kGroup * kSeg);
+#pragma unroll
+        for (int b = 0; b < kGroup; ++b)
+#pragma unroll
+            for (int k = 0; k < U; ++k)
+                f[b][k] = (ok && b < cnt) ? stage_field<BITS>(seg + b * (kSeg / 4), threadIdx.x + k * kDecThreads) : 0u;
+        if (q + S < n_steps) {
+            // every thread has taken its fields out of the stage: it may be refilled.  The same
+            // barrier makes the give-up decision uniform.
+            if (__syncthreads_or(!ok)) { expired = true; break; }
+            if (threadIdx.x == 0) issue(q + S);
+        } else if (!ok) {
+            expired = true;
+            break;
+        }
+#pragma unroll
+        for (int b = 0; b < kGroup; ++b) {
+            if (b < cnt) {           // uniform: only the last step of a worker count not divisible by kGroup is short
+#pragma unroll
+                for (int k = 0; k < U; ++k)
+                    add_unit<BITS>(acc[k], f[b][k], tab_bytes + b * (kTabStride * 4), i0 * (kTabStride * 4));
+            }
+        }
+    }
+    if (expired) {
+        atomicAdd(&g_wait_expired, 1u);
+        if (threadIdx.x == 0)      // the copies issued and not yet seen to land: steps q .. q + S - 1
+            for (uint32_t r = q; r < q + S && r < n_steps; ++r) mbar_wait(bar0 + 8 * (r % S), (r / S) & 1u);
+        return;
+    }
+
+    const uint64_t u0 = tile * Tile<BITS>::kUnits + threadIdx.x;
+    if (u0 * E >= d) return;       // nothing of this thread's first unit (hence of any) exists
+    finish_units<BITS, APPLY>(acc, u0, d, scale, divide, ap, out);
+}
+
+// Inputs of at least this many tiles go through the bulk-copy kernel; smaller ones are bound by
+// launch and set-up latency and keep the simpler direct kernel.
+constexpr uint64_t kBulkMinTiles = 8;
+
+template <int BITS, bool APPLY>
+static cudaError_t launch_bulk(const DecompressCall& c, const DecompressArgs& args, const DeviceTables& dt, float scale,
+                               int divide, const ApplyArgs& ap, uint64_t tiles) {
+    const size_t smem = static_cast<size_t>(c.n_workers) * (kTabStride * 4) +
+                        static_cast<size_t>(TQ_DECOMPRESS_STAGES) * kGroup * Tile<BITS>::kSegBytes + 16 + 8 * TQ_DECOMPRESS_STAGES;
+    if (smem > 48 * 1024) {
+        const cudaError_t e = cudaFuncSetAttribute(decompress_bulk_kernel<BITS, APPLY>,
+                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        if (e != cudaSuccess) return e;
+    }
+    decompress_bulk_kernel<BITS, APPLY><<<static_cast<unsigned>(tiles), kDecThreads, smem, c.stream>>>(
+        c.packed, c.words_stride, c.words_valid, c.n_workers, c.d, args, dt, scale, divide, ap, c.out);
+    return cudaGetLastError();
+}
+
 template <int BITS>
 static cudaError_t launch(const DecompressCall& c, const DecompressArgs& args, const DeviceTables& dt, float scale, int divide) {
     const uint64_t n_units = (c.d + Unit<BITS>::kElems - 1) / Unit<BITS>::kElems;
@@ -263,6 +445,9 @@ static cudaError_t launch(const DecompressCall& c, const DecompressArgs& args, c
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7FFFFFFFull) return cudaErrorInvalidConfiguration;
     const ApplyArgs ap{c.theta, c.momentum_buf, c.lr, c.mu, c.wd};
+    if (blocks >= kBulkMinTiles)
+        return c.theta ? launch_bulk<BITS, true>(c, args, dt, scale, divide, ap, blocks)
+                       : launch_bulk<BITS, false>(c, args, dt, scale, divide, ap, blocks);
     if (c.theta)
         decompress_kernel<BITS, true><<<static_cast<unsigned>(blocks), kDecThreads, 0, c.stream>>>(
             c.packed, c.words_stride, c.words_valid, c.n_workers, c.d, args, dt, scale, divide, ap, c.out);
@@ -270,6 +455,10 @@ static cudaError_t launch(const DecompressCall& c, const DecompressArgs& args, c
         decompress_kernel<BITS, false><<<static_cast<unsigned>(blocks), kDecThreads, 0, c.stream>>>(
             c.packed, c.words_stride, c.words_valid, c.n_workers, c.d, args, dt, scale, divide, ap, c.out);
     return cudaGetLastError();
+}
+
+cudaError_t read_wait_expired(unsigned int* count) {
+    return cudaMemcpyFromSymbol(count, g_wait_expired, sizeof(unsigned int));
 }
 
 cudaError_t launch_decompress(const DecompressCall& c) {

@@ -27,6 +27,7 @@ struct DecompressCall {
     float* theta = nullptr; float* momentum_buf = nullptr; float lr = 0.0f, mu = 0.0f, wd = 0.0f;   // fused model update
 };
 cudaError_t launch_decompress(const DecompressCall& c);
+cudaError_t read_wait_expired(unsigned int* count);   // give-ups of bounded barrier waits on the current device
 
 struct StatsCall {
     const void* grad; bool bf16; uint64_t d, grad_stride; uint32_t n_workers;

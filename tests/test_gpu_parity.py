@@ -208,7 +208,9 @@ def test_compress_caller_codebooks_grid_and_search_paths(tq, orc, dtype):
 def test_decompress_aggregate_exact(tq, orc, bits, n):
     L = 1 << bits
     rng = np.random.default_rng(bits * 100 + n)
-    for d in (1, 7, 8, 31, 32, 33, 255, 257, 4099, 100_003):
+    # up to 7 tiles of 4096 outputs: direct kernel; from 8 tiles on: bulk-copy kernel (whole tiles, one
+    # extra element, ragged tails)
+    for d in (1, 7, 8, 31, 32, 33, 255, 257, 4099, 28_672, 28_673, 32_768, 32_769, 65_535, 100_003):
         words = tq.tq_packed_words(d, bits)
         codes = rng.integers(0, L, (n, d), dtype=np.uint8)
         packed_h = np.stack([orc.pack(codes[i], bits) for i in range(n)])
@@ -523,3 +525,10 @@ def test_layer_groups_are_quantized_independently(tq, orc):
             assert np.array_equal(got[i], orc.compress(x, ops[i], 17, i))
         assert np.array_equal(out[lo:hi].cpu().numpy(), orc.decompress_aggregate(got, hi - lo, ops))
     assert max(alphas) > 5 * min(alphas)      # the groups really get different thresholds
+
+
+def test_no_bounded_wait_ran_out(tq):
+    """The bulk-copy decompression kernel gives up on a barrier after a fixed number of polls and counts
+    that; in a healthy run (everything above included, when run after it) the count is zero."""
+    torch.cuda.synchronize()
+    assert tq.tq_wait_expired_count() == 0
