@@ -280,9 +280,12 @@ decompress_kernel(const uint32_t* __restrict__ packed, uint64_t words_stride, ui
 // boundary and are a multiple of 16 bytes long (rows are padded to 16 bytes), as a bulk copy needs.
 // Every wait on a barrier is bounded; a wait that runs out makes the block count itself in
 // g_wait_expired, wait (bounded again) for its copies still in flight and return without storing.
-constexpr int kGroup = 4;                     // workers per stage
+#ifndef TQ_DECOMPRESS_GROUP
+#define TQ_DECOMPRESS_GROUP 4
+#endif
+constexpr int kGroup = TQ_DECOMPRESS_GROUP;   // workers per stage
 #ifndef TQ_DECOMPRESS_STAGES
-#define TQ_DECOMPRESS_STAGES 2
+#define TQ_DECOMPRESS_STAGES 3
 #endif
 constexpr uint32_t kWaitLimit = 1u << 22;     // polls of one barrier before giving up
 
@@ -328,8 +331,12 @@ __device__ __forceinline__ uint32_t stage_field(const uint32_t* seg, uint32_t ul
     }
 }
 
+#ifndef TQ_DECOMPRESS_BULK_BLOCKS
+#define TQ_DECOMPRESS_BULK_BLOCKS 8
+#endif
+
 template <int BITS, bool APPLY>
-__global__ void __launch_bounds__(kDecThreads, APPLY ? TQ_DECOMPRESS_MIN_BLOCKS - 2 : TQ_DECOMPRESS_MIN_BLOCKS)
+__global__ void __launch_bounds__(kDecThreads, APPLY ? TQ_DECOMPRESS_BULK_BLOCKS - 2 : TQ_DECOMPRESS_BULK_BLOCKS)
 decompress_bulk_kernel(const uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_valid, uint32_t n,
                        uint64_t d, const __grid_constant__ DecompressArgs args, const __grid_constant__ DeviceTables dt,
                        float scale, int divide, const __grid_constant__ ApplyArgs ap, float* __restrict__ out) {
