@@ -6,8 +6,8 @@
 // Work split: a thread owns 32 output elements as units whose codes fill whole 32-bit words (see
 // Unit below), keeps one fp32 accumulator per element in registers and walks the workers four at a
 // time so that many independent loads are in flight before the dependent lookups start.
-// Codebooks live in shared memory, 16 consecutive words per worker on a 256-byte pitch: any set of
-// codes of one worker maps to distinct banks, so lookups are conflict-free.
+// Codebooks live in shared memory, 16 consecutive words per worker, four workers per 256 bytes: any
+// set of codes of one worker maps to distinct banks, so lookups are conflict-free.
 // HBM traffic per output element: N * bits / 8 bytes read, 4 bytes written.
 #include "tq_device.cuh"
 #include "tq_launch.h"
@@ -37,7 +37,7 @@ __device__ __forceinline__ uint32_t ldg32_stream(const uint32_t* p) {
     return v;
 }
 
-constexpr int kTabStride = 64;   // floats between consecutive workers' codebooks in shared memory (256 bytes)
+constexpr int kTabStride = 16;   // floats between consecutive workers' codebooks in shared memory: four codebooks per 256 bytes
 
 // A unit is a run of elements decoded from one 32-bit "field": 8 / 16 / 32 elements = one packed word
 // for 4 / 2 / 1 bits; for 3 bits 8 elements = 24 bits that start on a byte boundary and are cut out of
@@ -84,7 +84,8 @@ __device__ __forceinline__ uint64_t last_word_of(uint64_t u) {
 }
 
 // Adds one worker's dequantized values for the E codes of field f to acc[0 .. E-1].  `tab_bytes + base`
-// is the worker's codebook in shared memory (base a multiple of 256).
+// is the worker's codebook in shared memory; base is a multiple of 256 (a group of four workers), the
+// worker's place in its group is part of tab_bytes.
 template <int BITS>
 __device__ __forceinline__ void add_unit(f32x2* acc, uint32_t f, const char* tab_bytes, uint32_t base) {
     constexpr int E = Unit<BITS>::kElems;
@@ -219,9 +220,10 @@ decompress_kernel(const uint32_t* __restrict__ packed, uint64_t words_stride, ui
                   float* __restrict__ out) {
     constexpr int E = Unit<BITS>::kElems, U = Unit<BITS>::kUnits;
 
-    // Each worker's codebook starts on a 256-byte boundary of shared memory, so a table offset
-    // (code * 4 < 64) can be merged into the worker's base offset by the same byte-permute that
-    // extracts it.  Bank = code: the lookups of one instruction never conflict.
+    // Every group of four codebooks starts on a 256-byte boundary of shared memory, so a table offset
+    // (code * 4 < 64) can be merged into the group's base offset by the same byte-permute that
+    // extracts it.  The lookups of one instruction go to one codebook, bank = code + 16 * (worker % 2):
+    // they never conflict.
     __shared__ __align__(256) float s_tab[TQ_MAX_WORKERS * kTabStride];
     fill_tables(s_tab, n, args, dt);
     __syncthreads();
@@ -264,7 +266,8 @@ decompress_kernel(const uint32_t* __restrict__ packed, uint64_t words_stride, ui
             f[k] = load_field_guarded<BITS>(packed + static_cast<uint64_t>(i) * words_stride,
                                             u0 + static_cast<uint64_t>(k) * kDecThreads, words_valid);
 #pragma unroll
-        for (int k = 0; k < U; ++k) add_unit<BITS>(acc[k], f[k], tab_bytes, i * (kTabStride * 4));
+        for (int k = 0; k < U; ++k)
+            add_unit<BITS>(acc[k], f[k], tab_bytes + (i & 3u) * (kTabStride * 4), (i & ~3u) * (kTabStride * 4));
     }
 
     finish_units<BITS, APPLY>(acc, u0, d, scale, divide, ap, out);
