@@ -119,7 +119,7 @@ def whole_job_gbs(world: int, bytes_per_rank: int, ms: float) -> float:
     return world * bytes_per_rank / (ms * 1e-3) / 1e9
 
 
-def cpu_oracle_round(w, sample_d: int, seed: int = 0):
+def cpu_oracle_round(w, sample_d: int, seed: int = 0, stats_rule: str = "hinted"):
     """One round of the path by the CPU oracle on `sample_d` elements per worker.  Returns seconds."""
     import numpy as np
     import torch
@@ -138,7 +138,7 @@ def cpu_oracle_round(w, sample_d: int, seed: int = 0):
     ps, rows = [], []
     for i, raw in enumerate(grads):
         x = oracle.bf16_to_f32(raw) if w.dtype == torch.bfloat16 else raw
-        st = oracle.stats(x)
+        st = oracle.stats_pow2(x) if stats_rule == "hinted" else oracle.stats(x)      # same g_min rule as the GPU arm
         p = oracle.params(st, w.num_levels, mode, w.gamma)
         ps.append(p)
         rows.append(oracle.compress(x, p, seed, i))
@@ -158,8 +158,8 @@ def run_reference(args, w):
     # bounded sample: about 1.5e9 element-rounds over the whole run (a couple of minutes of one core)
     sample_d = min(w.d, max(1 << 16, int(1.5e9 / max(args.steps + args.warmup, 1)) // w.n_workers))
     for _ in range(args.warmup):
-        cpu_oracle_round(w, sample_d)
-    times = [cpu_oracle_round(w, sample_d) for _ in range(args.steps)]
+        cpu_oracle_round(w, sample_d, stats_rule=args.stats)
+    times = [cpu_oracle_round(w, sample_d, stats_rule=args.stats) for _ in range(args.steps)]
     t = sum(times) / len(times)
     val = w.n_workers * sample_d * esz / t / 1e9
     sample = f"{w.n_workers} workers x {sample_d} elements of workload {w.name} per step (full round)"
@@ -187,6 +187,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--device-params", action="store_true",
                     help="design the parameters on the device (tq_params_device): no host round trip inside the round")
+    ap.add_argument("--stats", default="hinted", choices=["two-pass", "hinted"],
+                    help="two-pass: g_min = mean|g| (tq_stats); hinted: g_min = mean|g| rounded down to a power of two, "
+                         "one pass over the data with the previous round's mean as the hint (tq_stats_hinted)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -230,11 +233,18 @@ def main():
     stream = torch.cuda.current_stream()
 
     params_dev = torch.empty(N * 176, dtype=torch.uint8, device=dev)
+    hint = tq.new_gmin_hint(N, dev)
+
+    def run_stats(grad):
+        if args.stats == "hinted":
+            tq.tq_stats_hinted(grad, hint, d, stats_dev=stats_dev, workspace=ws)
+        else:
+            tq.tq_stats(grad, d, stats_dev=stats_dev, workspace=ws)
 
     def one_round(ev=None):
         """Returns what tq_decompress_aggregate needs to run again on this round's packed rows."""
         if ev: ev[0].record()
-        tq.tq_stats(g, d, stats_dev=stats_dev, workspace=ws)
+        run_stats(g)
         if ev: ev[1].record()
         if args.host_params:
             stats_pin.copy_(stats_dev, non_blocking=True)
@@ -290,8 +300,10 @@ def main():
     t_comp = statistics.mean(e[2].elapsed_time(e[3]) for e in evs)
     t_dec = statistics.mean(e[3].elapsed_time(e[4]) for e in evs)
     peak, peak_kind = hbm_peak()
+    stats_passes = 1 if args.stats == "hinted" else 2     # hinted: the second kernel returns at once when the hint holds
+    stats_key = "tq_stats (hinted, 1 pass)" if args.stats == "hinted" else "tq_stats (2 passes)"
     alg = {
-        "tq_stats (2 passes)": (2 * N * d * esz, t_stats, 2),
+        stats_key: (stats_passes * N * d * esz, t_stats, 2),
         "tq_compress": (N * d * esz + N * d * bits // 8, t_comp, 1),
         "tq_decompress_aggregate": (N * d * bits // 8 + 4 * d, t_dec, 1),
     }
@@ -334,7 +346,7 @@ def main():
 
         def e2e_round():
             g2.copy_(host_g, non_blocking=True)
-            tq.tq_stats(g2, d, stats_dev=stats_dev, workspace=ws)
+            run_stats(g2)
             if args.host_params:
                 stats_pin.copy_(stats_dev, non_blocking=True)
                 stream.synchronize()
@@ -363,7 +375,7 @@ def main():
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         sample_d = min(d, max(1 << 16, (1 << 26) // N))
-        dt = cpu_oracle_round(w, sample_d)
+        dt = cpu_oracle_round(w, sample_d, stats_rule=args.stats)
         cpu = {"value": N * sample_d * esz / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle", "seconds": dt,
                "host_cores_available": os.cpu_count(),
                "sample": f"{N} workers x {sample_d} elements of workload {w.name}, one full round"}
@@ -375,7 +387,10 @@ def main():
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "d": d, "n_workers": N, "mode": w.mode, "levels": w.num_levels, "bits": bits,
                        "gamma": w.gamma, "scale": w.scale, "storage": str(w.dtype).split(".")[-1],
-                       "g_min": "mean|g| per worker (two statistics passes)", "alpha_rule": "fixed point",
+                       "g_min": ("mean|g| per worker rounded down to a power of two; one statistics pass, hinted by the previous round's mean "
+                                 "(same data every round, so the hint always holds; when it does not, the tail pass runs again: --stats two-pass "
+                                 "shows that cost)" if args.stats == "hinted"
+                                 else "mean|g| per worker (two statistics passes)"), "alpha_rule": "fixed point",
                        "params": "host" if args.host_params else "device (no host round trip inside the round)",
                        "l2": f"inputs ({in_bytes / 1e6:.0f} MB) exceed L2; packed rows ({N * words * 4 / 1e6:.0f} MB) are "
                              "re-read right after being written, see kernels.tq_decompress_aggregate.cold_l2_*",

@@ -122,6 +122,33 @@ tq_status tq_stats(const void* grad_dev, tq_dtype dtype, uint64_t d, uint64_t gr
                    uint32_t n_workers, float g_min, float kappa, tq_stats_t* stats_dev,
                    void* workspace_dev, size_t ws_bytes, void* stream);
 
+/* What tq_stats_hinted remembers between rounds, one per worker, device memory owned by the caller.
+ * Zero-fill it before the first round. */
+typedef struct {
+    float level;     /* kappa * mean|g| of the last call (0: no hint yet) */
+    uint32_t hit;    /* 1: the last call's single pass already held the tail sums; 0: its tail pass had to run */
+} tq_gmin_hint_t;
+
+/*
+ * Statistics in ONE pass over the gradient, for the automatic threshold.
+ * Section 4.1 leaves the choice of g_min open ("the lower end of the power-law range"); this call
+ * uses g_min = kappa * mean|g| rounded DOWN to a power of two (0, i.e. no tail, below 2^-126).  A
+ * power-of-two threshold can be tried before the mean is known: the pass gathers the tail count and
+ * sum ln|g| for the two powers of two nearest to hint->level (the previous round's kappa * mean|g|),
+ * and when the finished mean selects one of them the record is complete after reading the data once.
+ * When it selects neither (first round; mean moved by more than a factor of about 1.4 to 2) a second
+ * kernel, which is always enqueued and otherwise returns at once, redoes the tail sums for the right
+ * threshold: the record is the same, bit for bit, either way, and the host never has to look.
+ *   hint_dev     [n_workers] tq_gmin_hint_t, device memory, 8-byte aligned, in/out (updated by every call).
+ *   kappa        > 0.
+ *   other arguments, the record's fields, workspace rules and errors as for tq_stats; stats_dev[i].g_min
+ *   is the power of two used.  tq_stats with that g_min passed explicitly gives the same counts (sums
+ *   to rounding).
+ */
+tq_status tq_stats_hinted(const void* grad_dev, tq_dtype dtype, uint64_t d, uint64_t grad_stride, uint32_t n_workers,
+                          float kappa, tq_gmin_hint_t* hint_dev, tq_stats_t* stats_dev, void* workspace_dev,
+                          size_t ws_bytes, void* stream);
+
 /*
  * tq_stats without a scratch argument, for callers that cannot allocate device memory.
  * (The paper has no counterpart; this is a packaging variant of tq_stats, same kernels, same results.)

@@ -82,6 +82,7 @@ def lib() -> C.CDLL:
         L.orc_rand16.argtypes = [u64, u32, u64]; L.orc_rand16.restype = u32
         L.orc_bf16_to_f32.argtypes = [C.c_void_p, u64, C.c_void_p]; L.orc_bf16_to_f32.restype = None
         L.orc_stats.argtypes = [C.c_void_p, u64, f32, f64, P(Stats)]; L.orc_stats.restype = i32
+        L.orc_pow2_floor.argtypes = [f32]; L.orc_pow2_floor.restype = f32
         for name in ("orc_model_pdf", "orc_model_QU", "orc_model_H", "orc_model_Hinv",
                      "orc_model_QN", "orc_truncation_bias"):
             fn = getattr(L, name); fn.argtypes = [P(Model), f64]; fn.restype = f64
@@ -163,6 +164,22 @@ def stats(g: np.ndarray, g_min: float = 0.0, kappa: float = 1.0) -> Stats:
     st = Stats()
     _check(lib().orc_stats(g.ctypes.data, g.size, g_min, kappa, C.byref(st)), "orc_stats")
     return st
+
+
+def pow2_floor(x: float) -> float:
+    return float(lib().orc_pow2_floor(C.c_float(x)))
+
+
+def stats_pow2(g: np.ndarray, kappa: float = 1.0) -> Stats:
+    """Statistics under the power-of-two threshold rule: g_min = pow2_floor((float)(kappa * mean|g|))."""
+    first = stats(g, 0.0, kappa)
+    g_min = pow2_floor(first.g_min)
+    if not g_min > 0.0:
+        first.g_min = 0.0
+        first.n_tail = 0
+        first.sum_log_tail = 0.0
+        return first
+    return stats(g, g_min, kappa)
 
 
 def params(st: Stats, num_levels: int, mode: int, gamma: float = math.nan,

@@ -61,6 +61,7 @@
  *   R13 aggregation: fp32 adds in worker order, then one IEEE division by N; with
  *       weights, each product w_i * v_i is rounded, then added, no division.
  */
+#include <float.h>
 #include <math.h>
 #include <stdint.h>
 #include <string.h>
@@ -165,6 +166,19 @@ int orc_stats(const float *g, uint64_t d, float g_min_in, double kappa, orc_stat
     }
     st->n_tail = n_tail; st->sum_log_tail = sum_log;
     return ORC_OK;
+}
+
+/* R19: the power-of-two threshold rule.  The largest power of two not above x, written with the
+ * C library's frexp / ldexp; 0 below the smallest normal float (no tail), Inf for Inf.
+ * The statistics under this rule are orc_stats called with g_min = orc_pow2_floor(kappa * mean|g|),
+ * the mean taken from a first orc_stats call (see stats_pow2 in the Python wrapper). */
+float orc_pow2_floor(float x)
+{
+    if (!(x >= FLT_MIN)) return 0.0f;
+    if (isinf(x)) return x;
+    int e;
+    (void)frexpf(x, &e);            /* x = m * 2^e, 0.5 <= m < 1 */
+    return ldexpf(0.5f, e);
 }
 
 /* ------------------------------------------------------------------------------------ */

@@ -25,7 +25,7 @@ UNIFORM, NONUNIFORM, BISCALED = 0, 1, 2
 ALPHA_CLOSED, ALPHA_FIXED_POINT, ALPHA_USER, ALPHA_MAXABS = 0, 1, 2, 3
 FLAG_ALPHA_CAPPED, FLAG_ALPHA_AT_GMIN, FLAG_GAMMA_FROM_MLE, FLAG_INVALID = 1, 2, 4, 8
 
-EXPORTS = ("tq_packed_words", "tq_stats_workspace_bytes", "tq_stats", "tq_stats_static", "tq_params", "tq_params_batch", "tq_params_from_levels", "tq_params_device",
+EXPORTS = ("tq_packed_words", "tq_stats_workspace_bytes", "tq_stats", "tq_stats_hinted", "tq_stats_static", "tq_params", "tq_params_batch", "tq_params_from_levels", "tq_params_device",
            "tq_compress_device_params", "tq_decompress_aggregate_device_params",
            "tq_compress", "tq_decompress_aggregate", "tq_decompress_aggregate_apply", "tq_strerror", "tq_last_cuda_error", "tq_kernel_launches", "tq_wait_expired_count")
 
@@ -70,6 +70,7 @@ def lib() -> C.CDLL:
         L.tq_packed_words.argtypes = [u64, u32]; L.tq_packed_words.restype = sz
         L.tq_stats_workspace_bytes.argtypes = [u32]; L.tq_stats_workspace_bytes.restype = sz
         L.tq_stats.argtypes = [vp, C.c_int, u64, u64, u32, f32, f32, vp, vp, sz, vp]; L.tq_stats.restype = C.c_int
+        L.tq_stats_hinted.argtypes = [vp, C.c_int, u64, u64, u32, f32, vp, vp, vp, sz, vp]; L.tq_stats_hinted.restype = C.c_int
         L.tq_stats_static.argtypes = [vp, C.c_int, u64, u64, u32, f32, f32, vp, vp]; L.tq_stats_static.restype = C.c_int
         L.tq_params.argtypes = [C.POINTER(Stats), u32, C.c_int, f64, C.c_int, f64, C.POINTER(Params)]
         L.tq_params.restype = C.c_int
@@ -161,6 +162,35 @@ def tq_stats(grad: torch.Tensor, d: Optional[int] = None, g_min: float = 0.0, ka
     _check(lib().tq_stats(grad.data_ptr(), _dtype_code(grad), d, stride, n, g_min, kappa, stats_dev.data_ptr(),
                           workspace.data_ptr(), workspace.numel(), _stream(stream)), "tq_stats")
     return stats_dev
+
+
+def tq_stats_hinted(grad: torch.Tensor, hint: torch.Tensor, d: Optional[int] = None, kappa: float = 1.0,
+                    stats_dev: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None, stream=None):
+    """One-pass statistics with g_min = kappa * mean|g| rounded down to a power of two.
+
+    ``hint`` is a device tensor of n_workers * 8 bytes (tq_gmin_hint_t records) that the caller keeps from
+    round to round; zero it before the first one (``new_gmin_hint``).  Returns the records' device tensor.
+    """
+    n, d, stride = _grad_layout(grad, d)
+    if stats_dev is None:
+        stats_dev = torch.empty(n * 64, dtype=torch.uint8, device=grad.device)
+    if workspace is None:
+        workspace = torch.empty(tq_stats_workspace_bytes(n), dtype=torch.uint8, device=grad.device)
+    _check(lib().tq_stats_hinted(grad.data_ptr(), _dtype_code(grad), d, stride, n, kappa, hint.data_ptr(),
+                                 stats_dev.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream(stream)),
+           "tq_stats_hinted")
+    return stats_dev
+
+
+def new_gmin_hint(n_workers: int, device="cuda") -> torch.Tensor:
+    """A zeroed hint buffer for tq_stats_hinted (n_workers records of {float level; uint32 hit})."""
+    return torch.zeros(n_workers * 8, dtype=torch.uint8, device=device)
+
+
+def gmin_hint_to_host(hint: torch.Tensor):
+    """[(level, hit)] per worker (synchronises)."""
+    raw = hint.cpu().numpy()
+    return list(zip(raw.view("<f4")[0::2].tolist(), raw.view("<u4")[1::2].tolist()))
 
 
 def tq_stats_static(grad: torch.Tensor, stats_dev: torch.Tensor, d: Optional[int] = None, g_min: float = 0.0,

@@ -36,6 +36,9 @@ struct StatsCall {
 // Enqueues the reduction; *launches receives the number of kernels launched.
 cudaError_t launch_stats(const StatsCall& c, int* launches);
 size_t stats_workspace_bytes(uint32_t n_workers);
+// One-pass reduction with a power-of-two threshold and a caller-kept hint, plus the tail pass that
+// runs only when the hint missed (two launches, the second usually returning at once).
+cudaError_t launch_stats_hinted(const StatsCall& c, tq_gmin_hint_t* hint, int* launches);
 // Same reduction with the library's built-in scratch array as workspace (c.workspace is ignored).
 // *limit is set when n_workers exceeds what the array holds; nothing is launched then.
 cudaError_t launch_stats_static(const StatsCall& c, int* launches, bool* limit);

@@ -102,6 +102,53 @@ def test_stats_parity(tq, orc, d, n, dtype):
                 assert math.isclose(s.sum_log_tail, ref.sum_log_tail, rel_tol=TOL_LOG, abs_tol=1e-9)
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("d,n", [(0, 1), (1, 1), (17, 3), (4099, 2), (100_003, 3), (3_000_000, 4)])
+def test_stats_hinted_parity_and_hint_independence(tq, orc, d, n, dtype):
+    """tq_stats_hinted against the oracle under the power-of-two threshold rule; the record must be the
+    same bit for bit whether the tail came from the single pass (hint hit) or from the second kernel
+    (no hint, stale hint)."""
+    g = heavy_tailed(d, n, dtype, seed=d + 3)
+    if d > 40:
+        g[:, 7] = float("nan"); g[:, 33] = float("inf"); g[0, 21] = float("-inf")
+    for kappa in (1.0, 2.5):
+        hint = tq.new_gmin_hint(n)
+        first = tq.tq_stats_hinted(g, hint, d, kappa=kappa).cpu().numpy().tobytes()       # no hint: second kernel
+        h1 = tq.gmin_hint_to_host(hint)
+        again = tq.tq_stats_hinted(g, hint, d, kappa=kappa).cpu().numpy().tobytes()       # hint from the same data
+        h2 = tq.gmin_hint_to_host(hint)
+        assert first == again
+        got = tq.stats_to_host(torch.frombuffer(bytearray(again), dtype=torch.uint8))
+        for i in range(n):
+            x = host_f32(orc, g[i, :d])
+            want = orc.stats_pow2(x, kappa=kappa)
+            s = got[i]
+            assert s.d == d and s.n_nonfinite == want.n_nonfinite and s.max_abs == want.max_abs
+            assert math.isclose(s.sum_abs, want.sum_abs, rel_tol=TOL_SUM, abs_tol=0)
+            assert math.isclose(s.sum_sq, want.sum_sq, rel_tol=TOL_SUM, abs_tol=0)
+            level = F32(kappa * s.sum_abs / d) if d else F32(0)
+            assert s.g_min == orc.pow2_floor(float(level))               # the rule, on the library's own mean
+            assert math.isclose(h2[i][0], float(level), rel_tol=1e-6, abs_tol=0) and h2[i][0] == h1[i][0]
+            assert h2[i][1] == 1 and h1[i][1] == (0 if s.g_min > 0 else 1)
+            if s.g_min == want.g_min:                                     # same binade as the oracle's mean (always, bar ties)
+                assert s.n_tail == want.n_tail
+                assert math.isclose(s.sum_log_tail, want.sum_log_tail, rel_tol=TOL_LOG, abs_tol=1e-9)
+        # a stale hint (mean moved by 8x): the second kernel runs again, same record
+        hint2 = tq.new_gmin_hint(n)
+        tq.tq_stats_hinted(g * 8 if dtype == torch.float32 else (g.float() * 8).to(dtype), hint2, d, kappa=kappa)
+        stale = tq.tq_stats_hinted(g, hint2, d, kappa=kappa).cpu().numpy().tobytes()
+        assert stale == first
+        if d > 40:
+            assert all(hit == 0 for _, hit in tq.gmin_hint_to_host(hint2))
+        # a hint one binade off still hits: candidates are the two powers of two nearest to it
+        hint3 = tq.new_gmin_hint(n)
+        tq.tq_stats_hinted((g.float() * 1.3).to(dtype), hint3, d, kappa=kappa)
+        near = tq.tq_stats_hinted(g, hint3, d, kappa=kappa).cpu().numpy().tobytes()
+        assert near == first
+        if d > 40:
+            assert all(hit == 1 for _, hit in tq.gmin_hint_to_host(hint3))
+
+
 def test_stats_is_deterministic_and_reuses_workspace(tq):
     g = heavy_tailed(1_000_003, 4, torch.float32, seed=3)
     ws = torch.empty(tq.tq_stats_workspace_bytes(4), dtype=torch.uint8, device="cuda")

@@ -324,6 +324,43 @@ def test_stats_match_numpy(orc):
     assert math.isclose(st3.g_min, 2 * st.g_min, rel_tol=1e-6)
 
 
+def test_pow2_floor_is_the_power_of_two_below(orc):
+    """The power-of-two threshold rule: pinned to 2^floor(log2 x) in float64 and to the bit pattern
+    (mantissa cleared); exact at powers of two, just below them, and at the edges of the normal range."""
+    rng = np.random.default_rng(12)
+    xs = np.exp(rng.uniform(np.log(1e-37), np.log(3e38), 2000)).astype(F32)
+    for x in xs:
+        want = 2.0 ** math.floor(math.log2(float(x)))
+        assert orc.pow2_floor(float(x)) == want
+        assert orc.pow2_floor(float(x)) == float((np.array([x]).view(np.uint32) & np.uint32(0xFF800000)).view(F32)[0])
+    for e in (-126, -20, -1, 0, 1, 30, 127):
+        p2 = float(F32(2.0) ** e)
+        assert orc.pow2_floor(p2) == p2
+        assert orc.pow2_floor(float(np.nextafter(F32(p2), F32(np.inf)))) == p2
+        if e > -126:
+            assert orc.pow2_floor(float(np.nextafter(F32(p2), F32(0)))) == p2 / 2
+    tiny = float(np.nextafter(F32(2.0) ** -126, F32(0)))            # largest subnormal: no tail
+    assert orc.pow2_floor(tiny) == 0.0 and orc.pow2_floor(0.0) == 0.0 and orc.pow2_floor(1e-45) == 0.0
+    assert orc.pow2_floor(float("inf")) == float("inf")
+
+
+def test_stats_under_the_power_of_two_rule(orc):
+    rng = np.random.default_rng(13)
+    for scale, kappa in ((1e-3, 1.0), (1e-3, 2.5), (3.0, 1.0), (1e-30, 1.0)):
+        g = (rng.standard_t(3.0, 50_001) * scale).astype(F32)
+        g[[3, 9]] = [np.nan, -np.inf]
+        plain = orc.stats(g, kappa=kappa)
+        st = orc.stats_pow2(g, kappa=kappa)
+        assert st.g_min <= plain.g_min < 2 * st.g_min and math.frexp(st.g_min)[0] == 0.5
+        assert (st.sum_abs, st.sum_sq, st.max_abs, st.n_nonfinite) == (plain.sum_abs, plain.sum_sq, plain.max_abs, plain.n_nonfinite)
+        fin = np.abs(g[np.isfinite(g)])
+        tail = fin[fin > F32(st.g_min)].astype(np.float64)
+        assert st.n_tail == tail.size >= plain.n_tail
+        assert math.isclose(st.sum_log_tail, np.log(tail / st.g_min).sum(), rel_tol=1e-11)
+    z = orc.stats_pow2(np.zeros(100, dtype=F32))
+    assert z.g_min == 0.0 and z.n_tail == 0 and z.sum_log_tail == 0.0
+
+
 def test_params_domain_errors(orc):
     st = orc.Stats(d=1000, n_tail=200, n_nonfinite=0, sum_abs=1.0, sum_sq=1.0, sum_log_tail=100.0,
                    max_abs=1.0, g_min=1e-3)
