@@ -457,7 +457,7 @@ static dim3 compress_grid(uint64_t d, uint32_t n_workers, bool persistent) {
     const uint64_t tiles = (n_runs + kThreads - 1) / kThreads;
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    uint64_t per_worker = (static_cast<uint64_t>(sms) * TQ_COMPRESS_MIN_BLOCKS + n_workers - 1) / n_workers;
+    uint64_t per_worker = static_cast<uint64_t>(sms) * TQ_COMPRESS_MIN_BLOCKS / n_workers;   // rounded down: one wave holds the grid
     if (!persistent || per_worker > tiles) per_worker = tiles;
     if (per_worker > 0x7FFFFFFFull) per_worker = 0x7FFFFFFFull;
     if (per_worker < 1) per_worker = 1;
