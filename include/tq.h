@@ -237,6 +237,20 @@ tq_status tq_decompress_aggregate(const uint32_t* packed_dev, size_t words_strid
                                   float* out_dev, void* stream);
 
 /*
+ * The same aggregation with the N packed rows given one by one (Algorithm 1, aggregation step, where
+ * worker i's message lives wherever worker i left it): rows_host[i] is the device address of worker
+ * i's packed row.  The rows need not be neighbours or share an allocation, and may be in another GPU's
+ * memory that the current device can read (peer access enabled, or a mapped symmetric buffer): the
+ * kernel then pulls each row's bytes straight over NVLink while it aggregates, with no gather copy
+ * first.  Every row: 16-byte aligned, at least tq_packed_words(d, bits) words readable.
+ *   rows_host    [n_workers] host array of device pointers; read during the call, not kept.
+ *   other arguments, arithmetic, result and errors as for tq_decompress_aggregate.
+ */
+tq_status tq_decompress_aggregate_rows(const uint32_t* const* rows_host, uint32_t n_workers, uint64_t d,
+                                       const tq_params_t* params_host, const float* weights_host, float* out_dev,
+                                       void* stream);
+
+/*
  * Server side including the model update (Algorithm 1, last step: theta <- theta - eta * g_bar) with the
  * optimiser of the paper's experiments (Section 5: momentum SGD with weight decay), fused into the
  * aggregation so that g_bar never goes to memory:

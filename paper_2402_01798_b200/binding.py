@@ -27,7 +27,7 @@ FLAG_ALPHA_CAPPED, FLAG_ALPHA_AT_GMIN, FLAG_GAMMA_FROM_MLE, FLAG_INVALID = 1, 2,
 
 EXPORTS = ("tq_packed_words", "tq_stats_workspace_bytes", "tq_stats", "tq_stats_hinted", "tq_stats_static", "tq_params", "tq_params_batch", "tq_params_from_levels", "tq_params_device",
            "tq_compress_device_params", "tq_decompress_aggregate_device_params",
-           "tq_compress", "tq_decompress_aggregate", "tq_decompress_aggregate_apply", "tq_strerror", "tq_last_cuda_error", "tq_kernel_launches", "tq_wait_expired_count")
+           "tq_compress", "tq_decompress_aggregate", "tq_decompress_aggregate_rows", "tq_decompress_aggregate_apply", "tq_strerror", "tq_last_cuda_error", "tq_kernel_launches", "tq_wait_expired_count")
 
 
 class Stats(C.Structure):
@@ -82,6 +82,8 @@ def lib() -> C.CDLL:
         L.tq_compress.restype = C.c_int
         L.tq_decompress_aggregate.argtypes = [vp, sz, u32, u64, C.POINTER(Params), C.POINTER(f32), vp, vp]
         L.tq_decompress_aggregate.restype = C.c_int
+        L.tq_decompress_aggregate_rows.argtypes = [C.POINTER(C.c_void_p), u32, u64, C.POINTER(Params), C.POINTER(f32), vp, vp]
+        L.tq_decompress_aggregate_rows.restype = C.c_int
         L.tq_params_device.argtypes = [vp, u32, u32, C.c_int, f64, C.c_int, f64, vp, vp]
         L.tq_params_device.restype = C.c_int
         L.tq_compress_device_params.argtypes = [vp, C.c_int, u64, u64, u32, vp, u32, C.c_int, u64, u32, vp, sz, vp]
@@ -273,6 +275,25 @@ def tq_decompress_aggregate(packed: torch.Tensor, d: int, params: Sequence[Param
     words_stride = packed.stride(0) if n > 1 else packed.shape[1]
     _check(lib().tq_decompress_aggregate(packed.data_ptr(), words_stride, n, d, _params_array(params), w,
                                          out.data_ptr(), _stream(stream)), "tq_decompress_aggregate")
+    return out
+
+
+def tq_decompress_aggregate_rows(rows: Sequence, d: int, params: Sequence[Params],
+                                 weights: Optional[Sequence[float]] = None, out: Optional[torch.Tensor] = None,
+                                 stream=None) -> torch.Tensor:
+    """tq_decompress_aggregate with one packed row per worker, each given as a 1-D int32 CUDA tensor or as a
+    raw device address (an int, e.g. a peer's buffer mapped into this process).  The caller keeps the rows
+    alive until the stream has passed the call."""
+    n = len(rows)
+    if len(params) != n:
+        raise ValueError("one Params per worker")
+    ptrs = (C.c_void_p * n)(*[int(r) if isinstance(r, int) else r.data_ptr() for r in rows])
+    if out is None:
+        dev = next((r.device for r in rows if not isinstance(r, int)), "cuda")
+        out = torch.empty(d, dtype=torch.float32, device=dev)
+    w = None if weights is None else (C.c_float * n)(*[float(x) for x in weights])
+    _check(lib().tq_decompress_aggregate_rows(ptrs, n, d, _params_array(params), w, out.data_ptr(), _stream(stream)),
+           "tq_decompress_aggregate_rows")
     return out
 
 

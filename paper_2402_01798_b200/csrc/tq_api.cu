@@ -143,6 +143,29 @@ tq_status tq_decompress_aggregate(const uint32_t* packed_dev, size_t words_strid
     return TQ_OK;
 }
 
+tq_status tq_decompress_aggregate_rows(const uint32_t* const* rows_host, uint32_t n_workers, uint64_t d,
+                                       const tq_params_t* params_host, const float* weights_host, float* out_dev,
+                                       void* stream) {
+    if (n_workers == 0 || n_workers > TQ_MAX_WORKERS || d > (1ull << 40)) return TQ_ERR_INVALID_ARG;
+    uint32_t bits = 0;
+    if (tq_status s = check_params(params_host, n_workers, &bits)) return s;
+    if (!rows_host || (d && !out_dev)) return TQ_ERR_INVALID_ARG;
+    for (uint32_t i = 0; i < n_workers; ++i) {
+        if (d && !rows_host[i]) return TQ_ERR_INVALID_ARG;
+        if (!aligned(rows_host[i], 16)) return TQ_ERR_ALIGNMENT;
+    }
+    if (!aligned(out_dev, 32)) return TQ_ERR_ALIGNMENT;
+    if (d == 0) return TQ_OK;
+    const size_t need = tq_packed_words(d, bits);
+    tq::DecompressCall c{nullptr, 0, need, n_workers, d, params_host, nullptr, weights_host, bits, out_dev,
+                         static_cast<cudaStream_t>(stream)};
+    c.rows = rows_host;
+    const cudaError_t e = tq::launch_decompress(c);
+    if (e != cudaSuccess) return cuda_failed(e);
+    g_launches += 1;
+    return TQ_OK;
+}
+
 tq_status tq_params_device(const tq_stats_t* stats_dev, uint32_t n_workers, uint32_t num_levels, tq_mode mode,
                            double gamma, tq_alpha_rule alpha_rule, double alpha_user, tq_params_t* params_dev,
                            void* stream) {

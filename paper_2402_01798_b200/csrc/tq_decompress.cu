@@ -25,6 +25,11 @@ struct ApplyArgs {
     float* momentum_buf;   // may be nullptr (no momentum)
     float lr, mu, wd;
 };
+// Where each worker's packed row starts.  Rows need not be neighbours, nor even live on this GPU: any
+// address the device can read (its own memory or a peer's mapped over NVLink) will do.
+struct RowTable {
+    const uint32_t* row[TQ_MAX_WORKERS];
+};
 struct DeviceTables {
     const tq_params_t* params_dev;    // nullptr: use DecompressArgs
     int use_weights;
@@ -214,7 +219,7 @@ __device__ __forceinline__ void fill_tables(float* s_tab, uint32_t n, const Deco
 
 template <int BITS, bool APPLY>
 __global__ void __launch_bounds__(kDecThreads, APPLY ? TQ_DECOMPRESS_MIN_BLOCKS - 2 : TQ_DECOMPRESS_MIN_BLOCKS)
-decompress_kernel(const uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_valid, uint32_t n,
+decompress_kernel(const __grid_constant__ RowTable rt, uint64_t words_valid, uint32_t n,
                   uint64_t d, const __grid_constant__ DecompressArgs args, const __grid_constant__ DeviceTables dt,
                   float scale, int divide, const __grid_constant__ ApplyArgs ap,
                   float* __restrict__ out) {
@@ -251,7 +256,7 @@ decompress_kernel(const uint32_t* __restrict__ packed, uint64_t words_stride, ui
             for (int b = 0; b < 4; ++b)
 #pragma unroll
                 for (int k = 0; k < U; ++k)
-                    f[b][k] = load_field<BITS>(packed + static_cast<uint64_t>(i + b) * words_stride, u0 + k * kDecThreads);
+                    f[b][k] = load_field<BITS>(rt.row[i + b], u0 + k * kDecThreads);
 #pragma unroll
             for (int b = 0; b < 4; ++b)
 #pragma unroll
@@ -263,7 +268,7 @@ decompress_kernel(const uint32_t* __restrict__ packed, uint64_t words_stride, ui
         uint32_t f[U];
 #pragma unroll
         for (int k = 0; k < U; ++k)
-            f[k] = load_field_guarded<BITS>(packed + static_cast<uint64_t>(i) * words_stride,
+            f[k] = load_field_guarded<BITS>(rt.row[i],
                                             u0 + static_cast<uint64_t>(k) * kDecThreads, words_valid);
 #pragma unroll
         for (int k = 0; k < U; ++k)
@@ -340,7 +345,7 @@ __device__ __forceinline__ uint32_t stage_field(const uint32_t* seg, uint32_t ul
 
 template <int BITS, bool APPLY>
 __global__ void __launch_bounds__(kDecThreads, APPLY ? TQ_DECOMPRESS_BULK_BLOCKS - 2 : TQ_DECOMPRESS_BULK_BLOCKS)
-decompress_bulk_kernel(const uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_valid, uint32_t n,
+decompress_bulk_kernel(const __grid_constant__ RowTable rt, uint64_t words_valid, uint32_t n,
                        uint64_t d, const __grid_constant__ DecompressArgs args, const __grid_constant__ DeviceTables dt,
                        float scale, int divide, const __grid_constant__ ApplyArgs ap, float* __restrict__ out) {
     constexpr int E = Unit<BITS>::kElems, U = Unit<BITS>::kUnits, S = TQ_DECOMPRESS_STAGES;
@@ -358,7 +363,6 @@ decompress_bulk_kernel(const uint32_t* __restrict__ packed, uint64_t words_strid
     const uint64_t row_bytes = words_valid * 4;
     const uint32_t seg_bytes = static_cast<uint32_t>(row_bytes - tile_off < kSeg ? row_bytes - tile_off : kSeg);
     const uint32_t n_steps = (n + kGroup - 1) / kGroup;
-    const char* src0 = reinterpret_cast<const char*>(packed) + tile_off;
 
     // step q = workers q*kGroup .. ; its bytes go to stage q % S
     auto issue = [&](uint32_t q) {
@@ -367,7 +371,7 @@ decompress_bulk_kernel(const uint32_t* __restrict__ packed, uint64_t words_strid
         const uint32_t bar = bar0 + 8 * st;
         mbar_expect_tx(bar, cnt * seg_bytes);
         for (uint32_t b = 0; b < cnt; ++b)
-            bulk_load(stage0 + (st * kGroup + b) * kSeg, src0 + static_cast<uint64_t>(i0 + b) * words_stride * 4, seg_bytes, bar);
+            bulk_load(stage0 + (st * kGroup + b) * kSeg, reinterpret_cast<const char*>(rt.row[i0 + b]) + tile_off, seg_bytes, bar);
     };
 
     if (threadIdx.x == 0) {
@@ -433,8 +437,8 @@ decompress_bulk_kernel(const uint32_t* __restrict__ packed, uint64_t words_strid
 constexpr uint64_t kBulkMinTiles = 8;
 
 template <int BITS, bool APPLY>
-static cudaError_t launch_bulk(const DecompressCall& c, const DecompressArgs& args, const DeviceTables& dt, float scale,
-                               int divide, const ApplyArgs& ap, uint64_t tiles) {
+static cudaError_t launch_bulk(const DecompressCall& c, const RowTable& rt, const DecompressArgs& args, const DeviceTables& dt,
+                               float scale, int divide, const ApplyArgs& ap, uint64_t tiles) {
     const size_t smem = static_cast<size_t>(c.n_workers) * (kTabStride * 4) +
                         static_cast<size_t>(TQ_DECOMPRESS_STAGES) * kGroup * Tile<BITS>::kSegBytes + 16 + 8 * TQ_DECOMPRESS_STAGES;
     if (smem > 48 * 1024) {
@@ -443,12 +447,13 @@ static cudaError_t launch_bulk(const DecompressCall& c, const DecompressArgs& ar
         if (e != cudaSuccess) return e;
     }
     decompress_bulk_kernel<BITS, APPLY><<<static_cast<unsigned>(tiles), kDecThreads, smem, c.stream>>>(
-        c.packed, c.words_stride, c.words_valid, c.n_workers, c.d, args, dt, scale, divide, ap, c.out);
+        rt, c.words_valid, c.n_workers, c.d, args, dt, scale, divide, ap, c.out);
     return cudaGetLastError();
 }
 
 template <int BITS>
-static cudaError_t launch(const DecompressCall& c, const DecompressArgs& args, const DeviceTables& dt, float scale, int divide) {
+static cudaError_t launch(const DecompressCall& c, const RowTable& rt, const DecompressArgs& args, const DeviceTables& dt, float scale,
+                          int divide) {
     const uint64_t n_units = (c.d + Unit<BITS>::kElems - 1) / Unit<BITS>::kElems;
     const uint64_t per_block = static_cast<uint64_t>(kDecThreads) * Unit<BITS>::kUnits;
     const uint64_t blocks = (n_units + per_block - 1) / per_block;
@@ -456,14 +461,14 @@ static cudaError_t launch(const DecompressCall& c, const DecompressArgs& args, c
     if (blocks > 0x7FFFFFFFull) return cudaErrorInvalidConfiguration;
     const ApplyArgs ap{c.theta, c.momentum_buf, c.lr, c.mu, c.wd};
     if (blocks >= kBulkMinTiles)
-        return c.theta ? launch_bulk<BITS, true>(c, args, dt, scale, divide, ap, blocks)
-                       : launch_bulk<BITS, false>(c, args, dt, scale, divide, ap, blocks);
+        return c.theta ? launch_bulk<BITS, true>(c, rt, args, dt, scale, divide, ap, blocks)
+                       : launch_bulk<BITS, false>(c, rt, args, dt, scale, divide, ap, blocks);
     if (c.theta)
         decompress_kernel<BITS, true><<<static_cast<unsigned>(blocks), kDecThreads, 0, c.stream>>>(
-            c.packed, c.words_stride, c.words_valid, c.n_workers, c.d, args, dt, scale, divide, ap, c.out);
+            rt, c.words_valid, c.n_workers, c.d, args, dt, scale, divide, ap, c.out);
     else
         decompress_kernel<BITS, false><<<static_cast<unsigned>(blocks), kDecThreads, 0, c.stream>>>(
-            c.packed, c.words_stride, c.words_valid, c.n_workers, c.d, args, dt, scale, divide, ap, c.out);
+            rt, c.words_valid, c.n_workers, c.d, args, dt, scale, divide, ap, c.out);
     return cudaGetLastError();
 }
 
@@ -474,6 +479,9 @@ cudaError_t read_wait_expired(unsigned int* count) {
 cudaError_t launch_decompress(const DecompressCall& c) {
     static thread_local DecompressArgs args;
     static thread_local DeviceTables dt;
+    static thread_local RowTable rt;
+    for (uint32_t i = 0; i < c.n_workers; ++i)
+        rt.row[i] = c.rows ? c.rows[i] : c.packed + static_cast<uint64_t>(i) * c.words_stride;
     dt.params_dev = c.params_dev;
     dt.use_weights = c.weights ? 1 : 0;
     for (uint32_t i = 0; i < c.n_workers; ++i) {
@@ -494,10 +502,10 @@ cudaError_t launch_decompress(const DecompressCall& c) {
         else { divide = 1; scale = static_cast<float>(n); }
     }
     switch (c.bits) {
-        case 1: return launch<1>(c, args, dt, scale, divide);
-        case 2: return launch<2>(c, args, dt, scale, divide);
-        case 3: return launch<3>(c, args, dt, scale, divide);
-        default: return launch<4>(c, args, dt, scale, divide);
+        case 1: return launch<1>(c, rt, args, dt, scale, divide);
+        case 2: return launch<2>(c, rt, args, dt, scale, divide);
+        case 3: return launch<3>(c, rt, args, dt, scale, divide);
+        default: return launch<4>(c, rt, args, dt, scale, divide);
     }
 }
 

@@ -25,6 +25,7 @@ struct DecompressCall {
     const float* weights; uint32_t bits;
     float* out; cudaStream_t stream;
     float* theta = nullptr; float* momentum_buf = nullptr; float lr = 0.0f, mu = 0.0f, wd = 0.0f;   // fused model update
+    const uint32_t* const* rows = nullptr;   // host array of n_workers row pointers; when set, packed / words_stride are unused
 };
 cudaError_t launch_decompress(const DecompressCall& c);
 cudaError_t read_wait_expired(unsigned int* count);   // give-ups of bounded barrier waits on the current device

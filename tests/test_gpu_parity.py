@@ -282,6 +282,40 @@ def test_decompress_aggregate_exact(tq, orc, bits, n):
             assert np.array_equal(gw, ww)
 
 
+@pytest.mark.parametrize("bits,n", [(4, 16), (3, 5), (2, 7), (1, 2)])
+def test_decompress_aggregate_rows_in_separate_allocations(tq, orc, bits, n):
+    """tq_decompress_aggregate_rows: every worker's row in its own allocation (offset inside it, given in a
+    shuffled order of allocation) gives the bytes of the contiguous call and of the oracle."""
+    L = 1 << bits
+    rng = np.random.default_rng(bits * 7 + n)
+    for d in (33, 4099, 100_003):
+        words = tq.tq_packed_words(d, bits)
+        codes = rng.integers(0, L, (n, d), dtype=np.uint8)
+        packed_h = np.stack([orc.pack(codes[i], bits) for i in range(n)])
+        ps = []
+        for i in range(n):
+            a = 0.01 * (1 + 0.3 * i)
+            mags = np.geomspace(a / 50, a, L // 2).astype(F32) if L > 2 else np.array([a], dtype=F32)
+            ps.append(tq.tq_params_from_levels([float(x) for x in np.concatenate([-mags[::-1], mags])]))
+        want = orc.decompress_aggregate(packed_h, d, [to_oracle_params(orc, p) for p in ps])
+        bufs = {}
+        for i in rng.permutation(n):                                  # allocation order != worker order
+            pad = 4 * int(rng.integers(0, 5))                          # 16-byte aligned offset into a larger buffer
+            buf = torch.full((pad + words + 8,), -1, dtype=torch.int32, device="cuda")
+            buf[pad:pad + words] = torch.from_numpy(packed_h[i].view(np.int32)).cuda()
+            bufs[int(i)] = (buf, pad)
+        rows = [bufs[i][0][bufs[i][1]:bufs[i][1] + words] for i in range(n)]
+        out = torch.full((d + 16,), 777.0, dtype=torch.float32, device="cuda")
+        tq.tq_decompress_aggregate_rows(rows, d, ps, out=out)
+        got = out.cpu().numpy()
+        assert np.array_equal(got[:d], want) and np.all(got[d:] == 777.0)
+        ptrs = [r.data_ptr() for r in rows]                            # raw addresses, as a peer mapping would give
+        got2 = tq.tq_decompress_aggregate_rows(ptrs, d, ps).cpu().numpy()
+        assert np.array_equal(got2, want)
+    with pytest.raises(tq.TqError):
+        tq.tq_decompress_aggregate_rows([rows[0].data_ptr() + 4] + rows[1:], d, ps)      # misaligned row
+
+
 # ------------------------------------------------------------------------------- whole round trips
 def run_round(tq, g, d, L, mode, gamma, seed):
     st, ps = lib_params_for(tq, g, d, L, mode, gamma)
