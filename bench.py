@@ -176,6 +176,97 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
+def run_exchange(args, w, tq, rank, local_rank, world, dev):
+    """The round with the N workers split over the ranks (strong scaling: the job is the same N x d whatever
+    the number of ranks).  Each rank takes the statistics of, and compresses, the workers it owns; the
+    64-byte statistics records and the packed rows are what crosses ranks; every rank forms the full update."""
+    import torch
+    import torch.distributed as dist
+    from paper_2402_01798_b200 import exchange, inputs
+    if not dist.is_initialized():
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29531")
+        dist.init_process_group("nccl", rank=0, world_size=1, device_id=dev)
+    esz = 2 if w.dtype == torch.bfloat16 else 4
+    mode = tq.NONUNIFORM if w.mode == "nonuniform" else tq.UNIFORM
+    N, d, bits = w.n_workers, w.d, w.bits
+    first, count = exchange.worker_slice(rank, world, N)
+    from dataclasses import replace
+    mine = replace(w, n_workers=max(count, 1), base_seed=w.base_seed + first)          # worker i's seed is base + i on any rank
+    g, stride = inputs.make_worker_gradients(mine, dev)
+    g = g[:count]
+    words = tq.tq_packed_words(d, bits)
+    stats_local = torch.zeros(max(count, 1) * 64, dtype=torch.uint8, device=dev)
+    ws = torch.empty(tq.tq_stats_workspace_bytes(max(count, 1)), dtype=torch.uint8, device=dev)
+    hint = tq.new_gmin_hint(max(count, 1), dev)
+    params_dev = torch.empty(N * 176, dtype=torch.uint8, device=dev)
+    out = torch.empty(d, dtype=torch.float32, device=dev)
+    peer = exchange.PeerRows(N, words, dev) if args.exchange == "peer" else None
+    packed_local = peer.local if peer else torch.empty((count, words), dtype=torch.int32, device=dev)
+
+    def one_round():
+        if count:
+            if args.stats == "hinted":
+                tq.tq_stats_hinted(g, hint, d, stats_dev=stats_local, workspace=ws)
+            else:
+                tq.tq_stats(g, d, stats_dev=stats_local, workspace=ws)
+        stats_all = exchange.gather_worker_rows(stats_local[: count * 64].view(count, 64), N)
+        tq.tq_params_device(stats_all.view(-1), N, w.num_levels, mode, w.gamma, params_dev=params_dev)
+        if args.exchange == "allgather":
+            if count:
+                tq.tq_compress_device_params(g, params_dev[first * 176:], w.num_levels, mode, seed=1234, first_worker=first,
+                                             d=d, packed=packed_local)
+            packed_all = exchange.gather_worker_rows(packed_local, N)
+            tq.tq_decompress_aggregate_device_params(packed_all, d, params_dev, w.num_levels, out=out)
+        else:
+            ps = tq.params_to_host(params_dev)                       # one host sync: the row-pointer call takes host records
+            if count:
+                tq.tq_compress(g, ps[first:first + count], seed=1234, first_worker=first, d=d, packed=packed_local)
+            peer.ready()                                              # every rank's rows are written ...
+            tq.tq_decompress_aggregate_rows(peer.row_addresses(), d, ps, out=out)
+            peer.done()                                               # ... and read, before the next round overwrites them
+
+    def barrier():
+        dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        one_round()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    l0 = tq.tq_kernel_launches()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    a.record()
+    for _ in range(args.steps):
+        one_round()
+    b.record()
+    barrier()
+    launches = tq.tq_kernel_launches() - l0
+    clocks = sampler.stop()
+    ms = max_over_ranks(a.elapsed_time(b), world, dev) / args.steps
+    checksum = float(out.double().sum().item())
+    if rank == 0:
+        peak, peak_kind = hbm_peak()
+        in_bytes = N * d * esz
+        line = {
+            "metric": METRIC, "value": in_bytes / (ms * 1e-3) / 1e9, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "d": d, "n_workers": N, "mode": w.mode, "levels": w.num_levels, "bits": bits,
+                       "gamma": w.gamma, "storage": str(w.dtype).split(".")[-1], "stats": args.stats,
+                       "multi_gpu": f"workers split over {world} rank(s), exchange = {args.exchange}: "
+                                    + ("statistics records and packed rows all-gathered over NCCL" if args.exchange == "allgather"
+                                       else "statistics records all-gathered, packed rows read in place from the peers' memory"),
+                       "exchanged_bytes_per_rank_per_step": int((N - count) * (words * 4 + 64))},
+            "roofline": None, "cpu_baseline": None, "e2e": None, "gpu_launches": int(launches), "clocks": clocks,
+            "update_checksum": checksum, "peak": {"hbm_gbs": peak, "source": peak_kind},
+        }
+        print(json.dumps(line), flush=True)
+    dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -190,6 +281,10 @@ def main():
     ap.add_argument("--stats", default="hinted", choices=["two-pass", "hinted"],
                     help="two-pass: g_min = mean|g| (tq_stats); hinted: g_min = mean|g| rounded down to a power of two, "
                          "one pass over the data with the previous round's mean as the hint (tq_stats_hinted)")
+    ap.add_argument("--exchange", default="replicas", choices=["replicas", "allgather", "peer"],
+                    help="replicas (default): every rank runs its own copy of the workload, nothing crosses ranks; "
+                         "allgather: the N workers are split over the ranks and the packed rows are all-gathered (NCCL) "
+                         "before the aggregation; peer: same split, the aggregation kernel reads the peers' rows in place")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -216,6 +311,9 @@ def main():
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     tq.lib()
+    if args.exchange != "replicas":
+        run_exchange(args, w, tq, rank, local_rank, world, dev)
+        return
 
     esz = 2 if w.dtype == torch.bfloat16 else 4
     mode = tq.NONUNIFORM if w.mode == "nonuniform" else tq.UNIFORM
@@ -398,6 +496,7 @@ def main():
             "hbm_frac_of_peak_whole_round": (sum(b for b, _, _ in alg.values()) / (ms_per_step * 1e-3) / 1e9) / peak,
             "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": int(launches), "clocks": clocks,
+            "update_checksum": float(out.double().sum().item()),      # rank 0's aggregated update, for comparing variants
         }
         print(json.dumps(line), flush=True)
     if world > 1:
