@@ -149,6 +149,22 @@ def test_stats_hinted_parity_and_hint_independence(tq, orc, d, n, dtype):
             assert all(hit == 1 for _, hit in tq.gmin_hint_to_host(hint3))
 
 
+def test_stats_hinted_degenerate_rows(tq, orc):
+    """All-zero and all-non-finite rows: no threshold (g_min = 0), no tail, and the hint says so."""
+    d = 5000
+    g = torch.zeros((3, d), dtype=torch.float32, device="cuda")
+    g[1, :] = float("nan")
+    g[2, ::2] = float("inf")
+    hint = tq.new_gmin_hint(3)
+    for _ in range(2):
+        st = tq.stats_to_host(tq.tq_stats_hinted(g, hint, d))
+        for i, bad in enumerate((0, d, d // 2)):
+            want = orc.stats_pow2(g[i].cpu().numpy())
+            assert (st[i].g_min, st[i].n_tail, st[i].sum_log_tail, st[i].n_nonfinite) == (0.0, 0, 0.0, bad)
+            assert (want.g_min, want.n_tail, want.n_nonfinite) == (0.0, 0, bad)
+        assert all(hit == 1 for _, hit in tq.gmin_hint_to_host(hint))
+
+
 def test_stats_is_deterministic_and_reuses_workspace(tq):
     g = heavy_tailed(1_000_003, 4, torch.float32, seed=3)
     ws = torch.empty(tq.tq_stats_workspace_bytes(4), dtype=torch.uint8, device="cuda")
