@@ -261,10 +261,11 @@ uint64_t tq_kernel_launches(void) { return g_launches.load(); }
 
 tq_status tq_wait_expired_count(uint32_t* count_host) {
     if (!count_host) return TQ_ERR_INVALID_ARG;
-    unsigned int n = 0;
-    const cudaError_t e = tq::read_wait_expired(&n);
+    unsigned int n = 0, m = 0;
+    cudaError_t e = tq::read_wait_expired(&n);
+    if (e == cudaSuccess) e = tq::read_compress_wait_expired(&m);
     if (e != cudaSuccess) return cuda_failed(e);
-    *count_host = n;
+    *count_host = n + m;
     return TQ_OK;
 }
 

@@ -17,6 +17,8 @@
 //     a saturating subtract of two exactly representable integers;
 //   - codes are kept as small floats and packed by exact multiply-adds (sums stay below 2^24);
 //   - table offsets are formed as denormal floats whose bit pattern IS the byte offset.
+#include <cuda.h>
+
 #include <cmath>
 
 #include "tq_device.cuh"
@@ -185,6 +187,10 @@ __device__ __forceinline__ float slot_as_float(const uint32_t (&rnd)[4], int e) 
     return __uint_as_float(__byte_perm(rnd[e >> 1], kMagicBits, (e & 1) ? 0x7432u : 0x7410u));
 }
 
+template <int BITS, int SEARCH, bool BF16, bool TAIL>
+__device__ __forceinline__ void quantize_run(const Raw8<BF16> (&g)[4], uint32_t* prow, uint64_t run, uint64_t d, uint64_t words_out,
+                                             uint32_t worker, const RoundKeys& rk, const RunCtx& cx);
+
 // One run of 32 elements: load, quantize, pack, store.  TAIL = the last, possibly partial run of a row
 // (element-wise guarded loads, zero padding bits, guarded stores and the row's alignment padding).
 template <int BITS, int SEARCH, bool BF16, bool TAIL>
@@ -206,6 +212,14 @@ __device__ __forceinline__ void compress_run(const char* row, uint32_t* prow, ui
             }
     }
 
+    quantize_run<BITS, SEARCH, BF16, TAIL>(g, prow, run, d, words_out, worker, rk, cx);
+}
+
+// The arithmetic of one run whose 32 elements are already in registers: quantize, pack, store.
+template <int BITS, int SEARCH, bool BF16, bool TAIL>
+__device__ __forceinline__ void quantize_run(const Raw8<BF16> (&g)[4], uint32_t* prow, uint64_t run, uint64_t d, uint64_t words_out,
+                                             uint32_t worker, const RoundKeys& rk, const RunCtx& cx) {
+    const uint64_t j0 = run << 5;
     const uint32_t blk_lo = static_cast<uint32_t>(j0 >> 3), blk_hi = static_cast<uint32_t>(j0 >> 35);
     const f32x2 alpha2 = both(cx.alpha), inv_step2 = both(cx.inv_step), cell_scale2 = both(cx.cell_scale);
     uint32_t chunk[4];   // the 8*BITS packed bits of each group
@@ -266,13 +280,10 @@ __device__ __forceinline__ void compress_run(const char* row, uint32_t* prow, ui
 #define TQ_COMPRESS_MIN_BLOCKS 4
 #endif
 
-// Per-block set-up of the shared tables for quantizer q, then the block's share of worker wi's runs.
+// Per-block set-up of the shared tables for quantizer q (ends with a block barrier unless SEARCH == kUniform).
 // s_grid must hold kMaxGridCells + 1 entries when SEARCH == kGrid.
-template <int BITS, int SEARCH, bool BF16>
-__device__ __forceinline__ void compress_block(const WorkerQ& q, float2* s_grid, float2* s_cell, float* s_search,
-                                               const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
-                                               const RoundKeys& rk, uint32_t worker, uint32_t wi,
-                                               uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_out) {
+template <int BITS, int SEARCH>
+__device__ __forceinline__ void build_tables(const WorkerQ& q, float2* s_grid, float2* s_cell, float* s_search) {
     constexpr int L = 1 << BITS;
     if constexpr (SEARCH != kUniform) {
         if (threadIdx.x < L - 1) s_cell[threadIdx.x] = make_float2(q.levels[threadIdx.x], q.inv_width[threadIdx.x]);
@@ -298,6 +309,16 @@ __device__ __forceinline__ void compress_block(const WorkerQ& q, float2* s_grid,
         }
     }
     if constexpr (SEARCH != kUniform) __syncthreads();
+}
+
+// Per-block set-up of the shared tables for quantizer q, then the block's share of worker wi's runs.
+// s_grid must hold kMaxGridCells + 1 entries when SEARCH == kGrid.
+template <int BITS, int SEARCH, bool BF16>
+__device__ __forceinline__ void compress_block(const WorkerQ& q, float2* s_grid, float2* s_cell, float* s_search,
+                                               const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
+                                               const RoundKeys& rk, uint32_t worker, uint32_t wi,
+                                               uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_out) {
+    build_tables<BITS, SEARCH>(q, s_grid, s_cell, s_search);
 
     constexpr size_t esz = BF16 ? 2 : 4;
     const char* row = static_cast<const char*>(grad) + static_cast<uint64_t>(wi) * grad_stride * esz;
@@ -327,6 +348,100 @@ compress_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
     const uint32_t wi = blockIdx.y;
     compress_block<BITS, SEARCH, BF16>(args.q[wi], s_grid, s_cell, s_search, grad, d, grad_stride, rk, first_worker + wi, wi,
                                        packed, words_stride, words_out);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Table-mode compress with the gradient tiles brought in by the tensor-memory accelerator.
+// A tile is 256 runs of 32 elements (one run per thread).  Thread 0 asks for the block's next tile as
+// ONE tiled copy ({32 elements, 256 runs, 1 worker} of the [N][runs][32] view of the gradient) while
+// the block is still quantizing the current one, so no warp waits on global loads and no registers are
+// held by loads in flight.  The copy lands swizzled (16-byte chunk c of run r at chunk c ^ (r & 7) for
+// 128-byte runs, c ^ ((r >> 1) & 3) for 64-byte runs), which makes a thread's reads of its own run
+// conflict-free.  Runs past the last whole run read as zeros and are not used; the row's last run
+// (possibly partial) goes through the guarded path.  Waits are bounded as in the header.
+__device__ unsigned int g_compress_wait_expired = 0;
+
+__device__ __forceinline__ void lds128(uint32_t addr, uint32_t& a, uint32_t& b, uint32_t& c, uint32_t& d) {
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(a), "=r"(b), "=r"(c), "=r"(d) : "r"(addr));
+}
+
+__device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y, int32_t z, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+
+template <int BITS, bool BF16>
+__global__ void __launch_bounds__(kThreads, TQ_COMPRESS_MIN_BLOCKS)
+compress_tma_kernel(const __grid_constant__ CUtensorMap tmap, const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
+                    const __grid_constant__ CompressArgs args, const __grid_constant__ RoundKeys rk,
+                    uint32_t first_worker, uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_out) {
+    constexpr uint32_t kRowBytes = 32 * (BF16 ? 2 : 4), kTileBytes = kThreads * kRowBytes;
+    __shared__ __align__(16) float2 s_grid[kMaxGridCells + 1];
+    __shared__ __align__(16) float2 s_cell[TQ_MAX_LEVELS];
+    extern __shared__ __align__(1024) unsigned char s_tile[];        // kTileBytes, then the barrier
+    const uint32_t wi = blockIdx.y;
+    const WorkerQ& q = args.q[wi];
+    const uint32_t tile0 = smem_addr(s_tile), bar = tile0 + kTileBytes;
+
+    const uint64_t n_runs = (d + 31) >> 5;
+    const uint64_t interior = n_runs - 1;                             // every run before the row's last one is whole
+    const uint32_t n_tiles = static_cast<uint32_t>((interior + kThreads - 1) / kThreads);
+    uint32_t tile = blockIdx.x;
+    auto issue = [&](uint32_t t) {
+        mbar_expect_tx(bar, kTileBytes);
+        tma_load_tile(tile0, &tmap, 0, static_cast<int32_t>(t * kThreads), static_cast<int32_t>(wi), bar);
+    };
+    if (threadIdx.x == 0) {
+        mbar_init(bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (tile < n_tiles) issue(tile);
+    }
+    build_tables<BITS, kGrid>(q, s_grid, s_cell, nullptr);            // ends with a block barrier
+
+    constexpr size_t esz = BF16 ? 2 : 4;
+    const char* row = static_cast<const char*>(grad) + static_cast<uint64_t>(wi) * grad_stride * esz;
+    uint32_t* prow = packed + static_cast<uint64_t>(wi) * words_stride;
+    const RunCtx cx{q.alpha, q.inv_step, q.top, q.inv_2alpha, q.cell_scale, reinterpret_cast<const char*>(s_grid),
+                    reinterpret_cast<const char*>(s_cell), nullptr};
+    // this thread's run starts at tile0 + tid * kRowBytes; its 16-byte chunk c sits at chunk c ^ sw: the chunk
+    // bits of the run's own address are zero, so the address of chunk c is (run | sw << 4) ^ (c << 4)
+    const uint32_t sw = BF16 ? ((threadIdx.x >> 1) & 3u) : (threadIdx.x & 7u);
+    const uint32_t mine0 = (tile0 + threadIdx.x * kRowBytes) | (sw << 4);
+
+    uint32_t parity = 0;
+    bool expired = false;
+    for (; tile < n_tiles; tile += gridDim.x) {
+        const bool ok = mbar_wait(bar, parity);
+        parity ^= 1u;
+        const uint64_t run = static_cast<uint64_t>(tile) * kThreads + threadIdx.x;
+        Raw8<BF16> g[4];         // read even if the wait ran out: the values are then never used
+#pragma unroll
+        for (int grp = 0; grp < 4; ++grp) {
+            if constexpr (BF16) {
+                lds128(mine0 ^ (static_cast<uint32_t>(grp) << 4), g[grp].v[0], g[grp].v[1], g[grp].v[2], g[grp].v[3]);
+            } else {
+                lds128(mine0 ^ (static_cast<uint32_t>(2 * grp) << 4), g[grp].v[0], g[grp].v[1], g[grp].v[2], g[grp].v[3]);
+                lds128(mine0 ^ (static_cast<uint32_t>(2 * grp + 1) << 4), g[grp].v[4], g[grp].v[5], g[grp].v[6], g[grp].v[7]);
+            }
+        }
+        // every thread has its run in registers: the tile buffer may be refilled.  The same barrier
+        // makes the give-up decision uniform.
+        if (__syncthreads_or(!ok)) { expired = true; break; }
+        if (threadIdx.x == 0 && tile + gridDim.x < n_tiles) issue(tile + gridDim.x);
+        if (run < interior) quantize_run<BITS, kGrid, BF16, false>(g, prow, run, d, words_out, first_worker + wi, rk, cx);
+    }
+    if (expired) {
+        atomicAdd(&g_compress_wait_expired, 1u);
+        if (threadIdx.x == 0) mbar_wait(bar, parity ^ 1u);            // the copy that did not land in time
+        return;
+    }
+    // the row's last run, by the thread that the striding would have given it to
+    if ((interior / kThreads) % gridDim.x == blockIdx.x && interior % kThreads == threadIdx.x)
+        compress_run<BITS, kGrid, BF16, true>(row, prow, interior, d, words_out, first_worker + wi, rk, cx);
+}
+
+cudaError_t read_compress_wait_expired(unsigned int* count) {
+    return cudaMemcpyFromSymbol(count, g_compress_wait_expired, sizeof(unsigned int));
 }
 
 // The grid cell of a value as a plain integer (device copy of the host's cell_of).
@@ -471,8 +586,65 @@ static cudaError_t launch(const CompressCall& c, const CompressArgs& args, dim3 
     return cudaGetLastError();
 }
 
+// ---- tiled copies: the tensor map of the gradient, [N][whole runs][32 elements] ------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+    static const EncodeTiledFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult how;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &how) != cudaSuccess ||
+            how != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// Inputs below this many elements per row keep the kernel that loads straight into registers.
+constexpr uint64_t kTmaMinElements = 1u << 16;
+
+// The map copies raw 32- or 16-bit words (no floating-point interpretation), rows past the last whole
+// run read as zeros.  Returns false when the tiled path does not apply (then the direct kernel runs).
+static bool make_tile_map(const CompressCall& c, CUtensorMap* map) {
+    const EncodeTiledFn encode = encode_tiled_fn();
+    const uint64_t whole = c.d / 32;
+    if (!encode || c.d < kTmaMinElements || whole > 0x7FFFFF00ull) return false;
+    const uint64_t esz = c.bf16 ? 2 : 4;
+    const cuuint64_t gdim[3] = {32, whole, c.n_workers};
+    const cuuint64_t row_pitch = c.n_workers > 1 ? c.grad_stride * esz : whole * 32 * esz;
+    const cuuint64_t gstride[2] = {32 * esz, row_pitch};              // bytes between runs, between workers
+    if (row_pitch % 16 != 0 || row_pitch >= (1ull << 40)) return false;
+    const cuuint32_t box[3] = {32, static_cast<cuuint32_t>(kThreads), 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = encode(map, c.bf16 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT32, 3,
+                              const_cast<void*>(c.grad), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                              c.bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+template <int BITS, bool BF>
+static cudaError_t launch_tma(const CompressCall& c, const CompressArgs& args, dim3 grid, const CUtensorMap& map) {
+    const int smem = kThreads * 32 * (BF ? 2 : 4) + 16;
+    const cudaError_t e = cudaFuncSetAttribute(compress_tma_kernel<BITS, BF>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    compress_tma_kernel<BITS, BF><<<grid, kThreads, smem, c.stream>>>(
+        map, c.grad, c.d, c.grad_stride, args, round_keys(c.seed), c.first_worker, c.packed, c.words_stride, c.words_out);
+    return cudaGetLastError();
+}
+
 template <int BITS>
 static cudaError_t dispatch(const CompressCall& c, const CompressArgs& a, dim3 grid, int search) {
+    // Tiled copies pay for bf16 rows (3 % faster at 124 M x 8: half the bytes per element, so the wait for
+    // global loads weighs more); for fp32 rows the kernel is bound by instruction issue and the extra
+    // shared-memory reads and the barrier per tile cost 2-3 %, so those keep the direct kernel.
+    if (search == kGrid && c.bf16) {
+        alignas(64) CUtensorMap map;
+        if (make_tile_map(c, &map)) return launch_tma<BITS, true>(c, a, grid, map);
+    }
     if (search == kGrid) return c.bf16 ? launch<BITS, kGrid, true>(c, a, grid) : launch<BITS, kGrid, false>(c, a, grid);
     if (search == kBinary) return c.bf16 ? launch<BITS, kBinary, true>(c, a, grid) : launch<BITS, kBinary, false>(c, a, grid);
     return c.bf16 ? launch<BITS, kUniform, true>(c, a, grid) : launch<BITS, kUniform, false>(c, a, grid);

@@ -295,7 +295,6 @@ constexpr int kGroup = TQ_DECOMPRESS_GROUP;   // workers per stage
 #ifndef TQ_DECOMPRESS_STAGES
 #define TQ_DECOMPRESS_STAGES 3
 #endif
-constexpr uint32_t kWaitLimit = 1u << 22;     // polls of one barrier before giving up
 
 __device__ unsigned int g_wait_expired = 0;   // blocks (or threads) whose bounded wait ran out, since load
 
@@ -305,28 +304,6 @@ struct Tile {
     static constexpr int kUnits = kDecThreads * Unit<BITS>::kUnits;     // units per tile (a multiple of 4)
     static constexpr int kSegBytes = kUnits * kUnitBytes;               // one worker's bytes per tile (a multiple of 16)
 };
-
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-// global -> this block's shared memory, `bytes` a multiple of 16, both addresses 16-byte aligned
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (uint32_t it = 0; it < kWaitLimit; ++it) {
-        uint32_t done;
-        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-        if (done) return true;
-    }
-    return false;
-}
 
 // The field of local unit ul of a tile segment in shared memory (same cut as load_field; the tile's
 // first unit is a multiple of 4, so the byte phase of a 3-bit unit is that of its local index).

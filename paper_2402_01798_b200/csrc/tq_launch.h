@@ -28,7 +28,8 @@ struct DecompressCall {
     const uint32_t* const* rows = nullptr;   // host array of n_workers row pointers; when set, packed / words_stride are unused
 };
 cudaError_t launch_decompress(const DecompressCall& c);
-cudaError_t read_wait_expired(unsigned int* count);   // give-ups of bounded barrier waits on the current device
+cudaError_t read_wait_expired(unsigned int* count);
+cudaError_t read_compress_wait_expired(unsigned int* count);   // the same for the tiled compress kernel   // give-ups of bounded barrier waits on the current device
 
 struct StatsCall {
     const void* grad; bool bf16; uint64_t d, grad_stride; uint32_t n_workers;

@@ -207,6 +207,36 @@ def test_compress_bit_exact_ragged_sizes(tq, orc, bits, mode, dtype):
             assert np.all(got[i, words:] == 0x5A5A5A5A)    # nothing written past the row's words
 
 
+@pytest.mark.parametrize("bits", [1, 2, 3, 4])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_compress_tiled_copy_path_ragged_sizes(tq, orc, bits, dtype):
+    """Table-mode bf16 rows of 65536 elements and more go through the kernel that brings the gradient in by
+    tiled copies (tiles of 8192 elements; fp32 rows keep the direct kernel and run here for comparison):
+    whole tiles, one run more or less, a partial last run, a last tile with a single run, several workers
+    with a padded row stride; salted with NaN, Inf, levels."""
+    L = 1 << bits
+    for d, n in ((65_536, 2), (65_537, 1), (65_568, 3), (73_728, 1), (73_729, 2), (81_919, 1), (200_003, 3)):
+        g = heavy_tailed(d, n, dtype, seed=7 * bits + d)
+        ps = []
+        for i in range(n):
+            s = orc.stats(host_f32(orc, g[i, :d]), g_min=5e-4)
+            ls = tq.Stats(d=s.d, n_tail=max(s.n_tail, 100), n_nonfinite=0, sum_abs=s.sum_abs, sum_sq=s.sum_sq,
+                          sum_log_tail=max(s.sum_log_tail, 50.0), max_abs=max(s.max_abs, 0.05), g_min=5e-4)
+            ps.append(tq.tq_params(ls, L, tq.NONUNIFORM, 3.0 + 0.25 * i))
+        salt_special_values(g, d, ps[0])
+        seed, first = 0x1234ABCD5678, 3
+        words = tq.tq_packed_words(d, bits)
+        packed = torch.full((n, words + 8), 0x5A5A5A5A, dtype=torch.int32, device="cuda")
+        tq.tq_compress(g, ps, seed, first, d=d, packed=packed)
+        got = packed.cpu().numpy().view(np.uint32)
+        for i in range(n):
+            want = orc.compress(host_f32(orc, g[i, :d]), to_oracle_params(orc, ps[i]), seed, first + i)
+            assert np.array_equal(got[i, :words], want), (d, i)
+            assert np.all(got[i, words:] == 0x5A5A5A5A)
+    torch.cuda.synchronize()
+    assert tq.tq_wait_expired_count() == 0
+
+
 @pytest.mark.parametrize("bits,mode", [(2, 0), (3, 1), (4, 1), (4, 0)])
 def test_compress_million_elements_and_seed_sensitivity(tq, orc, bits, mode):
     d, n = 1_000_000 + 37, 2
