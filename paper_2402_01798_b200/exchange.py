@@ -11,7 +11,7 @@ step).  This module holds what that needs on the host and nothing of the method'
     ``tq_decompress_aggregate`` runs on them;
   * ``PeerRows``: the packed rows placed in symmetric memory so that every rank can hand the peers' row
     ADDRESSES to ``tq_decompress_aggregate_rows``; the aggregation kernel then pulls each row over NVLink
-    while it aggregates and no gathered copy of the rows is ever written.  Plain (non-multicast) loads only.
+    while it aggregates and no gathered copy of the rows is ever written.  Every rank issues its own plain loads.
 
 Rows are always presented to the aggregation in global worker order, so the result does not depend on
 how many ranks there are.
