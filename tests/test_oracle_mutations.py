@@ -39,6 +39,8 @@ MUTATIONS = [
     ("biscaled inner mass", "double p1 = orc_model_QU(m, beta) / (2.0 * beta);", "double p1 = orc_model_QU(m, beta) / beta;", "test_oracle_biscaled.py"),
     ("update sign", "theta[j] = theta[j] - step;", "theta[j] = theta[j] + step;", "test_oracle_pack_aggregate.py"),
     ("momentum order", "float m = carried + g;", "float m = carried + lr * g;", "test_oracle_pack_aggregate.py"),
+    ("power of two rounded up", "return ldexpf(0.5f, e);", "return ldexpf(1.0f, e);", "test_oracle_params.py"),
+    ("power-of-two floor keeps subnormals", "if (!(x >= FLT_MIN)) return 0.0f;", "if (!(x > 0.0f)) return 0.0f;", "test_oracle_params.py"),
     ("cube root dropped", "double cb = cbrt((1.0 - 2.0 * m->rho) / (2.0 * m->g_min));\n    if (x <= m->g_min) return cb * x;", "double cb = (1.0 - 2.0 * m->rho) / (2.0 * m->g_min);\n    if (x <= m->g_min) return cb * x;", "test_oracle_params.py"),
 ]
 
