@@ -32,6 +32,40 @@ def test_library_exports_every_declared_symbol(tq):
         assert getattr(tq.lib(), name) is not None
 
 
+def test_header_is_plain_c_and_a_c_program_links(tq, tmp_path):
+    """include/tq.h compiles as C99 with warnings as errors, its structs have the documented sizes in C, and
+    a C program that calls only host-side entry points links against libtq.so and runs (no GPU needed)."""
+    import subprocess
+    src = tmp_path / "use_tq.c"
+    src.write_text(r"""
+#include <stdio.h>
+#include "tq.h"
+int main(void) {
+    tq_stats_t st = {0};
+    tq_params_t p;
+    tq_gmin_hint_t h = {0.0f, 0u};
+    (void)h;
+    if (sizeof(tq_stats_t) != 64 || sizeof(tq_params_t) != 176 || sizeof(tq_gmin_hint_t) != 8) return 2;
+    st.d = 1000000; st.n_tail = 200000; st.sum_abs = 1000.0; st.sum_sq = 4.0; st.sum_log_tail = 100000.0;
+    st.max_abs = 0.5f; st.g_min = 1e-3f;
+    if (tq_params(&st, 16, TQ_NONUNIFORM, 3.0, TQ_ALPHA_FIXED_POINT, 0.0, &p) != TQ_OK) return 3;
+    if (!(p.alpha > st.g_min) || p.num_levels != 16 || p.bits != 4) return 4;
+    if (tq_packed_words(100000, 2) != 6252) return 5;
+    if (tq_compress(NULL, TQ_F32, 10, 10, 1, &p, 1, 0, NULL, 0, NULL) == TQ_OK) return 6;   /* rejected before any CUDA call */
+    printf("%s\n", tq_strerror(TQ_ERR_ALIGNMENT));
+    return 0;
+}
+""")
+    exe = tmp_path / "use_tq"
+    inc = os.path.join(ROOT, "include")
+    libdir = os.path.dirname(tq.LIB_PATH)
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", inc, str(src), "-o", str(exe),
+                    "-L", libdir, "-ltq", "-Wl,-rpath," + libdir], check=True, capture_output=True)
+    r = subprocess.run([str(exe)], capture_output=True, text=True, timeout=120)
+    assert r.returncode == 0, (r.returncode, r.stderr)
+    assert "aligned" in r.stdout
+
+
 def test_missing_library_fails_loudly(tq, monkeypatch):
     monkeypatch.setattr(tq, "_lib", None)
     monkeypatch.setattr(tq, "LIB_PATH", os.path.join(ROOT, "no_such_dir", "libtq.so"))
