@@ -297,7 +297,7 @@ def test_compress_caller_codebooks_grid_and_search_paths(tq, orc, dtype):
 
 # ---------------------------------------------------------------------------- decompress-aggregate
 @pytest.mark.parametrize("bits", [1, 2, 3, 4])
-@pytest.mark.parametrize("n", [1, 2, 3, 5, 8, 16, 33])
+@pytest.mark.parametrize("n", [1, 2, 3, 5, 8, 16, 33, 64])
 def test_decompress_aggregate_exact(tq, orc, bits, n):
     L = 1 << bits
     rng = np.random.default_rng(bits * 100 + n)
