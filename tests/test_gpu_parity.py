@@ -208,10 +208,11 @@ def test_compress_bit_exact_ragged_sizes(tq, orc, bits, mode, dtype):
 
 
 @pytest.mark.parametrize("bits", [1, 2, 3, 4])
+@pytest.mark.parametrize("mode", [0, 1])
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
-def test_compress_tiled_copy_path_ragged_sizes(tq, orc, bits, dtype):
+def test_compress_tiled_copy_path_ragged_sizes(tq, orc, bits, mode, dtype):
     """Table-mode bf16 rows of 65536 elements and more go through the kernel that brings the gradient in by
-    tiled copies (tiles of 8192 elements; fp32 rows keep the direct kernel and run here for comparison):
+    tiled copies (tiles of 8192 elements; fp32 rows and uniform mode keep the direct kernel and run here too):
     whole tiles, one run more or less, a partial last run, a last tile with a single run, several workers
     with a padded row stride; salted with NaN, Inf, levels."""
     L = 1 << bits
@@ -222,7 +223,7 @@ def test_compress_tiled_copy_path_ragged_sizes(tq, orc, bits, dtype):
             s = orc.stats(host_f32(orc, g[i, :d]), g_min=5e-4)
             ls = tq.Stats(d=s.d, n_tail=max(s.n_tail, 100), n_nonfinite=0, sum_abs=s.sum_abs, sum_sq=s.sum_sq,
                           sum_log_tail=max(s.sum_log_tail, 50.0), max_abs=max(s.max_abs, 0.05), g_min=5e-4)
-            ps.append(tq.tq_params(ls, L, tq.NONUNIFORM, 3.0 + 0.25 * i))
+            ps.append(tq.tq_params(ls, L, mode, 3.0 + 0.25 * i))
         salt_special_values(g, d, ps[0])
         seed, first = 0x1234ABCD5678, 3
         words = tq.tq_packed_words(d, bits)
