@@ -322,7 +322,7 @@ def test_decompress_aggregate_exact(tq, orc, bits, n):
         assert np.all(np.abs(got[:d] - want) <= 1e-6 * np.maximum(np.abs(got[:d]), np.abs(want)))
         assert np.array_equal(got[:d], want)
         assert np.all(got[d:] == 777.0)                    # no write past d
-        if n in (3, 8) and d in (33, 4099):
+        if n in (3, 8, 33) and d in (33, 4099, 100_003):
             w = rng.random(n).astype(F32); w /= w.sum()
             gw = tq.tq_decompress_aggregate(packed, d, ps, weights=list(w)).cpu().numpy()
             ww = orc.decompress_aggregate(packed_h, d, [to_oracle_params(orc, p) for p in ps], weights=w)
