@@ -210,6 +210,21 @@ def test_argument_validation_without_a_gpu(tq):
     assert L.tq_stats(ok_ptr, tq.F32, 64, 64, 2, 0.0, 0.0, ok_ptr, ok_ptr, ws, None) == tq.ERR_INVALID_ARG
     assert L.tq_stats(ok_ptr, tq.F32, 64, 64, 2, 0.0, 1.0, None, ok_ptr, ws, None) == tq.ERR_INVALID_ARG
     assert L.tq_stats(ok_ptr, tq.F32, 64, 64, 2, 0.0, 1.0, ok_ptr, ok_ptr + 8, ws, None) == tq.ERR_ALIGNMENT
+    # one-pass statistics: hint pointer, kappa, workspace
+    assert L.tq_stats_hinted(ok_ptr, tq.F32, 64, 64, 2, 1.0, None, ok_ptr, ok_ptr, ws, None) == tq.ERR_INVALID_ARG
+    assert L.tq_stats_hinted(ok_ptr, tq.F32, 64, 64, 2, 0.0, ok_ptr, ok_ptr, ok_ptr, ws, None) == tq.ERR_INVALID_ARG
+    assert L.tq_stats_hinted(ok_ptr, tq.F32, 64, 64, 2, float("inf"), ok_ptr, ok_ptr, ok_ptr, ws, None) == tq.ERR_INVALID_ARG
+    assert L.tq_stats_hinted(ok_ptr, tq.F32, 64, 64, 2, 1.0, ok_ptr + 4, ok_ptr, ok_ptr, ws, None) == tq.ERR_ALIGNMENT
+    assert L.tq_stats_hinted(ok_ptr, tq.F32, 64, 64, 2, 1.0, ok_ptr, ok_ptr, ok_ptr, ws - 1, None) == tq.ERR_BUFFER_TOO_SMALL
+    # aggregation over row pointers: null table, null row, misaligned row, misaligned output
+    rows = (C.c_void_p * 2)(ok_ptr, ok_ptr + 4096)
+    assert L.tq_decompress_aggregate_rows(None, 2, 64, arr, None, ok_ptr, None) == tq.ERR_INVALID_ARG
+    assert L.tq_decompress_aggregate_rows((C.c_void_p * 2)(ok_ptr, None), 2, 64, arr, None, ok_ptr, None) == tq.ERR_INVALID_ARG
+    assert L.tq_decompress_aggregate_rows((C.c_void_p * 2)(ok_ptr, ok_ptr + 8), 2, 64, arr, None, ok_ptr, None) == tq.ERR_ALIGNMENT
+    assert L.tq_decompress_aggregate_rows(rows, 2, 64, arr, None, ok_ptr + 16, None) == tq.ERR_ALIGNMENT
+    assert L.tq_decompress_aggregate_rows(rows, 2, 64, mixed, None, ok_ptr, None) == tq.ERR_INVALID_ARG
+    assert L.tq_decompress_aggregate_rows(rows, 2, 0, arr, None, ok_ptr, None) == tq.OK
+    assert L.tq_wait_expired_count(None) == tq.ERR_INVALID_ARG
     # d = 0 needs no device at all
     assert L.tq_compress(ok_ptr, tq.F32, 0, 0, 1, arr, 0, 0, ok_ptr, 0, None) == tq.OK
     assert L.tq_decompress_aggregate(ok_ptr, 0, 1, 0, arr, None, ok_ptr, None) == tq.OK
