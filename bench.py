@@ -409,6 +409,19 @@ def main():
     kernels.update({k: {"ms": t, "launches_per_step": n, "algorithmic_bytes": b, "gbs": b / (t * 1e-3) / 1e9,
                    "frac_of_hbm_peak": b / (t * 1e-3) / 1e9 / peak} for k, (b, t, n) in alg.items()})
 
+    if args.stats == "hinted":
+        # what the statistics cost when the hint does not hold (first round, or the mean moved to another binade):
+        # the tail kernel then reads the data a second time
+        miss = []
+        for _ in range(3):
+            hint.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); run_stats(g); b.record()
+            torch.cuda.synchronize()
+            miss.append(a.elapsed_time(b))
+        kernels[stats_key]["hint_miss_ms"] = statistics.mean(miss)
+        run_stats(g)                                     # leave a valid hint behind
+
     # decompress-aggregate again with the packed rows evicted from L2 first (in the round above they
     # were just written by tq_compress, so part of them is still cache-resident)
     decompress_again = one_round()
