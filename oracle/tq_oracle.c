@@ -60,6 +60,11 @@
  *       Section 5: g += wd*theta; m = mu*m + g; theta -= lr*m; fp32, each operation rounded once.
  *   R13 aggregation: fp32 adds in worker order, then one IEEE division by N; with
  *       weights, each product w_i * v_i is rounded, then added, no division.
+ *   R14 non-finite gradients: counted by the statistics and left out of every sum; the quantizer
+ *       sends NaN to -alpha (code 0) and +-Inf to +-alpha (fmaxf / fminf semantics).
+ *   R15 uniform index: x = (t + alpha) * inv_step in fp32, two roundings; k = min(floor x, s-1).
+ *   R19 one-pass statistics: the automatic threshold kappa * mean|g| is rounded DOWN to a power of
+ *       two (0, i.e. no tail, below the smallest normal number): orc_pow2_floor, orc_stats_pow2.
  */
 #include <float.h>
 #include <math.h>

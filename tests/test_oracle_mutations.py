@@ -41,6 +41,8 @@ MUTATIONS = [
     ("momentum order", "float m = carried + g;", "float m = carried + lr * g;", "test_oracle_pack_aggregate.py"),
     ("power of two rounded up", "return ldexpf(0.5f, e);", "return ldexpf(1.0f, e);", "test_oracle_params.py"),
     ("power-of-two floor keeps subnormals", "if (!(x >= FLT_MIN)) return 0.0f;", "if (!(x > 0.0f)) return 0.0f;", "test_oracle_params.py"),
+    ("bf16 widening shift", "uint32_t bits = (uint32_t)in[i] << 16;", "uint32_t bits = (uint32_t)in[i] << 15;", "test_oracle_load_window.py"),
+    ("window index off by one", "orc_code_at(q, g[i], seed, worker, j0 + i);", "orc_code_at(q, g[i], seed, worker, j0 + i + 1);", "test_oracle_load_window.py"),
     ("cube root dropped", "double cb = cbrt((1.0 - 2.0 * m->rho) / (2.0 * m->g_min));\n    if (x <= m->g_min) return cb * x;", "double cb = (1.0 - 2.0 * m->rho) / (2.0 * m->g_min);\n    if (x <= m->g_min) return cb * x;", "test_oracle_params.py"),
 ]
 
