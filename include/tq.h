@@ -108,8 +108,8 @@ size_t tq_stats_workspace_bytes(uint32_t n_workers);
  * Section 4.1: rho = tail mass beyond g_min).  One 64-byte record per worker.
  *   grad_dev     [n_workers][grad_stride] elements of `dtype`, 32-byte aligned; worker i's slice is
  *                the first d elements of row i.  grad_stride (elements) must keep rows 32-byte aligned.
- *   g_min        > 0: threshold for the tail.  <= 0: each worker uses kappa * mean|g| of its own
- *                slice (one extra pass over the data).
+ *   g_min        > 0: threshold for the tail (any positive fp32 value, subnormal ones included).
+ *                <= 0: each worker uses kappa * mean|g| of its own slice (one extra pass over the data).
  *   stats_dev    [n_workers] tq_stats_t, device memory, 8-byte aligned; valid when the stream reaches
  *                the end of this call's work (copy it back to the host for tq_params).
  *   workspace_dev, ws_bytes   device scratch of at least tq_stats_workspace_bytes(n_workers), 256-byte
@@ -131,7 +131,8 @@ typedef struct {
 
 /*
  * Statistics in ONE pass over the gradient, for the automatic threshold.
- * Section 4.1 leaves the choice of g_min open ("the lower end of the power-law range"); this call
+ * Section 4.1 introduces g_min only as the point from which the power-law behaviour holds and gives no
+ * rule for choosing it; this call
  * uses g_min = kappa * mean|g| rounded DOWN to a power of two (0, i.e. no tail, below 2^-126).  A
  * power-of-two threshold can be tried before the mean is known: the pass gathers the tail count and
  * sum ln|g| for the two powers of two nearest to hint->level (the previous round's kappa * mean|g|),
@@ -169,6 +170,10 @@ tq_status tq_stats_hinted(const void* grad_dev, tq_dtype dtype, uint64_t d, uint
  * contents: the library clears the ticket counters itself at the start of every call, nothing else
  * needs to start at zero.  Two calls whose kernels overlap on the same GPU (different streams, or
  * different host threads) race on the array and give wrong statistics: serialise them.
+ * The looked-up address is remembered per device ordinal for the life of the process.  It does not
+ * survive cudaDeviceReset, nor a second CUDA context on the same ordinal: a process that resets a device
+ * or switches contexts must not call tq_stats_static on that device afterwards (use tq_stats with its
+ * own workspace there).
  */
 tq_status tq_stats_static(const void* grad_dev, tq_dtype dtype, uint64_t d, uint64_t grad_stride,
                           uint32_t n_workers, float g_min, float kappa, tq_stats_t* stats_dev, void* stream);
@@ -229,8 +234,9 @@ tq_status tq_compress(const void* grad_dev, tq_dtype dtype, uint64_t d, uint64_t
  * Server side (Algorithm 1, aggregation step): out_j = sum_i w_i * levels_i[code_ij].
  *   weights_host NULL: w_i = 1/N (Lemma 2): fp32 adds in worker order, then one division by N.
  *                else [n_workers] fp32: each product is rounded, then added in worker order.
- *   out_dev      [d] fp32, 16-byte aligned.
- * Errors: INVALID_ARG, ALIGNMENT, BUFFER_TOO_SMALL, CUDA.
+ *   out_dev      [d] fp32, 32-byte aligned (the kernel stores 32 bytes per thread at a time).
+ * Errors: INVALID_ARG, ALIGNMENT, BUFFER_TOO_SMALL, CUDA.  TQ_OK means the launch was accepted; it does
+ * not cover a bounded wait running out inside the kernel, see tq_wait_expired_count.
  */
 tq_status tq_decompress_aggregate(const uint32_t* packed_dev, size_t words_stride, uint32_t n_workers,
                                   uint64_t d, const tq_params_t* params_host, const float* weights_host,
@@ -258,6 +264,10 @@ tq_status tq_decompress_aggregate_rows(const uint32_t* const* rows_host, uint32_
  *     m_j = momentum * m_j + g  (when momentum_dev is given; g = m_j);  theta_j -= lr * g.
  * fp32, every operation rounded once.  theta_dev [d] and momentum_dev [d] (may be NULL) are fp32 device
  * arrays, 32-byte aligned, updated in place.  Other arguments and errors as tq_decompress_aggregate.
+ * A tile whose bounded wait ran out (see tq_wait_expired_count) is left as it was, so after such a launch
+ * theta and the momentum buffer are updated in some tiles and not in others: a caller that cannot
+ * tolerate that checks tq_wait_expired_count before and after the step and restores theta from its own
+ * copy when the count moved.
  */
 tq_status tq_decompress_aggregate_apply(const uint32_t* packed_dev, size_t words_stride, uint32_t n_workers, uint64_t d,
                                         const tq_params_t* params_host, const float* weights_host, float* theta_dev,
@@ -297,7 +307,9 @@ uint64_t tq_kernel_launches(void); /* kernels launched by this library in this p
 
 /* Bounded waits.  The large-input decompression kernel stages packed bytes through asynchronous bulk
  * copies and waits for them on shared-memory barriers; every such wait gives up after a fixed number
- * of polls.  A block whose wait ran out stores nothing for its tile and counts itself here.
+ * of polls.  A block whose wait ran out stores nothing for the tile it was working on (the decision is
+ * taken by the whole block, so a tile is never partly stored), abandons its remaining tiles and counts
+ * itself here.
  * *count_host receives the number of such give-ups on the current device since the library was loaded
  * (0 in a healthy run: a non-zero value means the outputs of the affected launch are incomplete).
  * Synchronises the device.  Returns TQ_ERR_INVALID_ARG for a null pointer, TQ_ERR_CUDA if the read fails.

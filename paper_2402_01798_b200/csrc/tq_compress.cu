@@ -15,6 +15,8 @@
 //   - threshold T = rint(p * 2^16): one fused multiply-add with 2^23;
 //   - the random slot r as the float 2^23 + r: one byte-permute; [r < T] = sat((2^23 + T) - (2^23 + r)),
 //     a saturating subtract of two exactly representable integers;
+//   - uniform codebook: interval and threshold together as the one integer X = rint(x * 2^16) = k * 2^16 + T,
+//     code = ceil((X - r) / 2^16), with the clamps of x done by saturating multiplies and subtracts;
 //   - codes are kept as small floats and packed by exact multiply-adds (sums stay below 2^24);
 //   - table offsets are formed as denormal floats whose bit pattern IS the byte offset.
 #include <cuda.h>
@@ -32,6 +34,7 @@ constexpr int kMinGridCells = 32;
 // Per-worker quantizer as the kernel sees it.
 struct WorkerQ {
     float alpha, inv_step, top;   // top = (float)(L-1)
+    float inv_step_l;             // inv_step / L when that quotient is exact and normal, else 0 (uniform mode)
     float inv_2alpha;             // maps [-alpha, alpha] to [0, 1] for the lookup grid
     float cell_scale;             // grid cells M as the denormal M * 2^-149
     uint32_t cells;               // M
@@ -42,7 +45,10 @@ struct CompressArgs {
     WorkerQ q[TQ_MAX_WORKERS];
 };
 
-enum Search { kUniform = 0, kGrid = 1, kBinary = 2 };
+// kUniformWide: the uniform codebook through the arithmetic that needs no scaled inverse step (used
+// only when inv_step / L would be subnormal, i.e. alpha beyond about 2^121).
+enum Search { kUniform = 0, kGrid = 1, kBinary = 2, kUniformWide = 3 };
+__host__ __device__ constexpr bool is_uniform(int search) { return search == kUniform || search == kUniformWide; }
 
 cudaError_t launch_compress_dev(const CompressCall& c);
 
@@ -71,20 +77,62 @@ __device__ __forceinline__ float rounds_up(float p, float rf) {
 }
 
 // Uniform codebook, l_k = -alpha + k * 2 alpha / s (Section 4.1), two elements at a time.  Reference
-// form of the decision: t = clip(g), x = (t + alpha) * inv_step, k = min(floor x, s-1), p = x - k.
-// Computed here as x = clip((g + alpha) * inv_step, 0, s), k' = floor x, p' = x - k': the affine map is
-// monotone, so clipping after it gives the same x for |g| <= alpha and 0 / >= s beyond; at x = s this
-// yields k' = s, p' = 0, i.e. the same code s as k = s-1, p >= 1.  NaN becomes 0 (fmaxf drops it).
-__device__ __forceinline__ f32x2 code_uniform2(float g0, float g1, f32x2 alpha2, f32x2 inv_step2, float top,
-                                               float rf0, float rf1) {
+// form of the decision: t = clip(g), x = (t + alpha) * inv_step, k = min(floor x, s-1), p = x - k,
+// T = rint(p * 2^16), code = k + [r < T].
+//
+// Computed here through the single integer X = rint(x * 2^16): since k * 2^16 is an integer,
+// X = k * 2^16 + T (a carry when T = 2^16 is the next interval with T = 0, the same code), and
+// code = k + [r < T] = ceil((X - r) / 2^16) for 0 <= r < 2^16.  With L = s + 1 a power of two:
+//   sum = g + alpha                            (as the reference; for |g| <= alpha it is t + alpha)
+//   y   = sat(sum * (inv_step / L))            = clip(x, 0, L) / L exactly: scaling by a power of two commutes
+//                                                with the rounding of the product, and .sat sends NaN and
+//                                                negatives to 0, which is where the reference sends them
+//   y  -= sat(y - s/L)                         = min(y, s/L): for y in (s/L, 1] the difference is exact
+//                                                (s/L >= 1/2, Sterbenz), so the result is s/L itself; this is
+//                                                x = s, which the reference codes as s, like every g >= alpha
+//   Xm  = fma(y, L * 2^16, 2^23)               = 2^23 + X, rounded to nearest-even as rint does (2^23 is even)
+//   v   = Xm - (2^23 + r)                      = X - r, exact
+//   cm  = fma.rp(v, 2^-16, 1.5 * 2^23)         = 1.5 * 2^23 + ceil(v / 2^16): the sum stays inside one binade
+// and the caller subtracts the bias (or most of it, see pack8).  sum0 / sum1 are g + alpha of the pair.
+struct UniformQ {
+    float inv_step_l, c_top;      // inv_step / L, s / L
+    f32x2 scale2;                 // L * 2^16, twice
+};
+constexpr float kCodeBias = 12582912.0f;                 // 1.5 * 2^23
+__device__ __forceinline__ f32x2 fma2_ru(f32x2 a, f32x2 b, f32x2 c) {   // round toward +infinity
+    f32x2 r; asm("fma.rp.f32x2 %0, %1, %2, %3;" : "=l"(r.v) : "l"(a.v), "l"(b.v), "l"(c.v)); return r;
+}
+__device__ __forceinline__ f32x2 code_uniform2(float sum0, float sum1, const UniformQ& u, float rf0, float rf1) {
+    const float y0 = mul_sat(sum0, u.inv_step_l), y1 = mul_sat(sum1, u.inv_step_l);
+    const f32x2 y = sub2(pair(y0, y1), pair(sub_sat(y0, u.c_top), sub_sat(y1, u.c_top)));
+    const f32x2 v = sub2(fma2(y, u.scale2, both(kMagic)), pair(rf0, rf1));
+    return fma2_ru(v, both(1.52587890625e-5f), both(kCodeBias));
+}
+
+// The same decision without the scaled inverse step (alpha so large that inv_step / L is subnormal):
+// x = clip((g + alpha) * inv_step, 0, s), k' = floor x, p' = x - k'; at x = s this yields k' = s, p' = 0,
+// i.e. the same code s as k = s-1, p >= 1.  NaN becomes 0 (fmaxf drops it).  Returns the plain code.
+__device__ __forceinline__ f32x2 code_uniform2_wide(float sum0, float sum1, f32x2 inv_step2, float top, float rf0, float rf1) {
     float x0, x1;
-    unpair(mul2(add2(pair(g0, g1), alpha2), inv_step2), x0, x1);
+    unpair(mul2(pair(sum0, sum1), inv_step2), x0, x1);
     const f32x2 x = pair(fminf(fmaxf(x0, 0.0f), top), fminf(fmaxf(x1, 0.0f), top));
     const f32x2 magic2 = both(kMagic);
     const f32x2 kf = sub2(add2_rd(x, magic2), magic2);                       // floor(x), exact
     float pm0, pm1;
     unpair(fma2(sub2(x, kf), both(65536.0f), magic2), pm0, pm1);            // 2^23 + rint(p * 2^16)
     return add2(kf, pair(sub_sat(pm0, rf0), sub_sat(pm1, rf1)));
+}
+
+// g + alpha for elements 2h and 2h+1 of a loaded group.  bf16 storage: the widening is part of the add
+// (the stored 16 bits are an exact fp32 value, so the sum rounds as the fp32 add of the widened value).
+template <bool BF16>
+__device__ __forceinline__ void pair_plus_alpha(const Raw8<BF16>& g, int h, float alpha, float& sum0, float& sum1) {
+    if constexpr (BF16) {
+        asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tadd.rn.f32.bf16 %0, lo, %3;\n\tadd.rn.f32.bf16 %1, hi, %3;\n\t}"
+            : "=f"(sum0), "=f"(sum1) : "r"(g.v[h]), "f"(alpha));
+    } else {
+        unpair(add2(pair(__uint_as_float(g.v[2 * h]), __uint_as_float(g.v[2 * h + 1])), both(alpha)), sum0, sum1);
+    }
 }
 
 // General codebook through the lookup grid, two elements at a time.  s_grid[c] = (boundary, k_lo): k_lo
@@ -131,22 +179,40 @@ __device__ __forceinline__ float code_binary(float g, float alpha, const float* 
 
 // Four pairs of float codes (elements 0..7 of a group, each code < 2^BITS) -> their 8*BITS packed
 // bits, LSB first.  Every partial sum is an integer below 2^24, so the fp32 arithmetic is exact.
-template <int BITS>
+// Returns a word whose low 8*BITS bits are the packed codes; with BIASED (2- and 4-bit codes only) the
+// bits above them are not zero and the caller merges chunks by byte-permutes.
+//
+// BIASED: the caller left 2^23 in the even element of pair 0 (and of pair 2 for 4-bit codes), see
+// code_bias().  The 16-bit partial results then appear as 2^23 + value, whose bit pattern holds the
+// value in its low half, and no float -> integer conversion is needed.
+template <int BITS, bool BIASED>
 __device__ __forceinline__ uint32_t pack8(const f32x2 (&c)[4]) {
     constexpr float B = static_cast<float>(1 << BITS), B2 = B * B;
+    static_assert(!BIASED || BITS == 2 || BITS == 4, "only 16-bit partial results fit beside the bias");
     if constexpr (BITS <= 3) {
         f32x2 a = fma2(c[3], both(B2), c[2]);
         a = fma2(a, both(B2), c[1]);
         a = fma2(a, both(B2), c[0]);
         float ev, od;
         unpair(a, ev, od);
-        return __float2uint_rz(__fmaf_rn(od, B, ev));
+        if constexpr (BIASED) return __float_as_uint(__fmaf_rn(od, B, ev));   // 2^23 + 16 bits
+        else return __float2uint_rz(__fmaf_rn(od, B, ev));
     } else {
         float e0, o0, e1, o1;
         unpair(fma2(c[1], both(B2), c[0]), e0, o0);       // elements 0..3: 16 bits
         unpair(fma2(c[3], both(B2), c[2]), e1, o1);       // elements 4..7: 16 bits
-        return __float2uint_rz(__fmaf_rn(o0, B, e0)) + (__float2uint_rz(__fmaf_rn(o1, B, e1)) << 16);
+        if constexpr (BIASED)
+            return __byte_perm(__float_as_uint(__fmaf_rn(o0, B, e0)), __float_as_uint(__fmaf_rn(o1, B, e1)), 0x5410u);
+        else return __float2uint_rz(__fmaf_rn(o0, B, e0)) + (__float2uint_rz(__fmaf_rn(o1, B, e1)) << 16);
     }
+}
+// What to subtract from code_uniform2's result for pair h of a group so that pack8<BITS, BIASED> can
+// take it: the whole bias 1.5 * 2^23, except 2^22 in the even element of the pairs that start a 16-bit
+// partial result, which therefore keeps 2^23.
+template <int BITS, bool BIASED>
+__device__ __forceinline__ f32x2 code_bias(int h) {
+    const bool keep = BIASED && (h == 0 || (BITS == 4 && h == 2));
+    return pair(keep ? 4194304.0f : kCodeBias, kCodeBias);
 }
 
 // The ten Philox round keys (key advanced by the Weyl constants), computed once on the host: they
@@ -179,8 +245,22 @@ __device__ __forceinline__ void philox_rounds(uint32_t c0, uint32_t c1, uint32_t
 
 struct RunCtx {
     float alpha, inv_step, top, inv_2alpha, cell_scale;
+    UniformQ u;
     const char* s_grid; const char* s_cell; const float* s_search;
 };
+
+template <int BITS>
+__device__ __forceinline__ UniformQ uniform_q(const WorkerQ& q) {
+    constexpr float L = static_cast<float>(1 << BITS);
+    return UniformQ{q.inv_step_l, (L - 1.0f) / L, both(L * 65536.0f)};
+}
+
+// inv_step / L for the scaled uniform path: exact when the quotient is a normal number (L is a power of
+// two); 0 tells the launch to use the unscaled arithmetic instead.  Same expression on host and device.
+__host__ __device__ inline float scaled_inv_step(float inv_step, uint32_t num_levels) {
+    const float q = inv_step / static_cast<float>(num_levels);
+    return (q >= 1.17549435e-38f && q <= 3.402823466e38f) ? q : 0.0f;
+}
 
 // the 16 random bits of slot e of a Philox block, as the float 2^23 + r
 __device__ __forceinline__ float slot_as_float(const uint32_t (&rnd)[4], int e) {
@@ -222,6 +302,8 @@ __device__ __forceinline__ void quantize_run(const Raw8<BF16> (&g)[4], uint32_t*
     const uint64_t j0 = run << 5;
     const uint32_t blk_lo = static_cast<uint32_t>(j0 >> 3), blk_hi = static_cast<uint32_t>(j0 >> 35);
     const f32x2 alpha2 = both(cx.alpha), inv_step2 = both(cx.inv_step), cell_scale2 = both(cx.cell_scale);
+    // whole runs of the scaled uniform path hand pack8 biased codes (2- and 4-bit codes)
+    constexpr bool BIASED = SEARCH == kUniform && !TAIL && (BITS == 2 || BITS == 4);
     uint32_t chunk[4];   // the 8*BITS packed bits of each group
 #pragma unroll
     for (int grp = 0; grp < 4; ++grp) {
@@ -232,12 +314,18 @@ __device__ __forceinline__ void quantize_run(const Raw8<BF16> (&g)[4], uint32_t*
         for (int h = 0; h < 4; ++h) {            // elements 2h, 2h+1 of the group
             const int e = 2 * h;
             const float rf0 = slot_as_float(rnd, e), rf1 = slot_as_float(rnd, e + 1);
-            const float g0 = elem<BF16>(g[grp], e), g1 = elem<BF16>(g[grp], e + 1);
-            if constexpr (SEARCH == kUniform) code[h] = code_uniform2(g0, g1, alpha2, inv_step2, cx.top, rf0, rf1);
-            else if constexpr (SEARCH == kGrid)
-                code[h] = code_grid2(g0, g1, alpha2, cx.inv_2alpha, cell_scale2, cx.s_grid, cx.s_cell, rf0, rf1);
-            else code[h] = pair(code_binary<BITS>(g0, cx.alpha, cx.s_search, reinterpret_cast<const float2*>(cx.s_cell), rf0),
-                                code_binary<BITS>(g1, cx.alpha, cx.s_search, reinterpret_cast<const float2*>(cx.s_cell), rf1));
+            if constexpr (is_uniform(SEARCH)) {
+                float sum0, sum1;
+                pair_plus_alpha<BF16>(g[grp], h, cx.alpha, sum0, sum1);
+                if constexpr (SEARCH == kUniform) code[h] = sub2(code_uniform2(sum0, sum1, cx.u, rf0, rf1), code_bias<BITS, BIASED>(h));
+                else code[h] = code_uniform2_wide(sum0, sum1, inv_step2, cx.top, rf0, rf1);
+            } else {
+                const float g0 = elem<BF16>(g[grp], e), g1 = elem<BF16>(g[grp], e + 1);
+                if constexpr (SEARCH == kGrid)
+                    code[h] = code_grid2(g0, g1, alpha2, cx.inv_2alpha, cell_scale2, cx.s_grid, cx.s_cell, rf0, rf1);
+                else code[h] = pair(code_binary<BITS>(g0, cx.alpha, cx.s_search, reinterpret_cast<const float2*>(cx.s_cell), rf0),
+                                    code_binary<BITS>(g1, cx.alpha, cx.s_search, reinterpret_cast<const float2*>(cx.s_cell), rf1));
+            }
             if constexpr (TAIL) {                 // padding bits are zero
                 float c0, c1;
                 unpair(code[h], c0, c1);
@@ -246,7 +334,7 @@ __device__ __forceinline__ void quantize_run(const Raw8<BF16> (&g)[4], uint32_t*
                 code[h] = pair(c0, c1);
             }
         }
-        chunk[grp] = pack8<BITS>(code);
+        chunk[grp] = pack8<BITS, BIASED>(code);
     }
 
     // four chunks of 8*BITS bits -> BITS words, LSB first
@@ -257,7 +345,7 @@ __device__ __forceinline__ void quantize_run(const Raw8<BF16> (&g)[4], uint32_t*
         w[1] = (chunk[1] >> 8) | (chunk[2] << 16);
         w[2] = (chunk[2] >> 16) | (chunk[3] << 8);
     }
-    if constexpr (BITS == 2) { w[0] = chunk[0] | (chunk[1] << 16); w[1] = chunk[2] | (chunk[3] << 16); }
+    if constexpr (BITS == 2) { w[0] = __byte_perm(chunk[0], chunk[1], 0x5410u); w[1] = __byte_perm(chunk[2], chunk[3], 0x5410u); }
     if constexpr (BITS == 1) { w[0] = chunk[0] | (chunk[1] << 8) | (chunk[2] << 16) | (chunk[3] << 24); }
 
     uint32_t* dst = prow + run * BITS;
@@ -280,12 +368,12 @@ __device__ __forceinline__ void quantize_run(const Raw8<BF16> (&g)[4], uint32_t*
 #define TQ_COMPRESS_MIN_BLOCKS 4
 #endif
 
-// Per-block set-up of the shared tables for quantizer q (ends with a block barrier unless SEARCH == kUniform).
+// Per-block set-up of the shared tables for quantizer q (ends with a block barrier unless the codebook is uniform).
 // s_grid must hold kMaxGridCells + 1 entries when SEARCH == kGrid.
 template <int BITS, int SEARCH>
 __device__ __forceinline__ void build_tables(const WorkerQ& q, float2* s_grid, float2* s_cell, float* s_search) {
     constexpr int L = 1 << BITS;
-    if constexpr (SEARCH != kUniform) {
+    if constexpr (!is_uniform(SEARCH)) {
         if (threadIdx.x < L - 1) s_cell[threadIdx.x] = make_float2(q.levels[threadIdx.x], q.inv_width[threadIdx.x]);
     }
     if constexpr (SEARCH == kBinary) {
@@ -308,7 +396,7 @@ __device__ __forceinline__ void build_tables(const WorkerQ& q, float2* s_grid, f
             s_grid[c] = make_float2(boundary, below);
         }
     }
-    if constexpr (SEARCH != kUniform) __syncthreads();
+    if constexpr (!is_uniform(SEARCH)) __syncthreads();
 }
 
 // Per-block set-up of the shared tables for quantizer q, then the block's share of worker wi's runs.
@@ -324,7 +412,7 @@ __device__ __forceinline__ void compress_block(const WorkerQ& q, float2* s_grid,
     const char* row = static_cast<const char*>(grad) + static_cast<uint64_t>(wi) * grad_stride * esz;
     uint32_t* prow = packed + static_cast<uint64_t>(wi) * words_stride;
     const uint64_t n_runs = (d + 31) >> 5;
-    const RunCtx cx{q.alpha, q.inv_step, q.top, q.inv_2alpha, q.cell_scale, reinterpret_cast<const char*>(s_grid),
+    const RunCtx cx{q.alpha, q.inv_step, q.top, q.inv_2alpha, q.cell_scale, uniform_q<BITS>(q), reinterpret_cast<const char*>(s_grid),
                     reinterpret_cast<const char*>(s_cell), s_search};
     const uint64_t stride = static_cast<uint64_t>(gridDim.x) * kThreads;
 
@@ -401,7 +489,7 @@ compress_tma_kernel(const __grid_constant__ CUtensorMap tmap, const void* __rest
     constexpr size_t esz = BF16 ? 2 : 4;
     const char* row = static_cast<const char*>(grad) + static_cast<uint64_t>(wi) * grad_stride * esz;
     uint32_t* prow = packed + static_cast<uint64_t>(wi) * words_stride;
-    const RunCtx cx{q.alpha, q.inv_step, q.top, q.inv_2alpha, q.cell_scale, reinterpret_cast<const char*>(s_grid),
+    const RunCtx cx{q.alpha, q.inv_step, q.top, q.inv_2alpha, q.cell_scale, uniform_q<BITS>(q), reinterpret_cast<const char*>(s_grid),
                     reinterpret_cast<const char*>(s_cell), nullptr};
     // this thread's run starts at tile0 + tid * kRowBytes; its 16-byte chunk c sits at chunk c ^ sw: the chunk
     // bits of the run's own address are zero, so the address of chunk c is (run | sw << 4) ^ (c << 4)
@@ -471,6 +559,7 @@ __device__ __forceinline__ void load_worker(const tq_params_t* __restrict__ para
         const float inv_2alpha = ok ? __fdiv_rn(1.0f, __fmul_rn(2.0f, alpha)) : 0.0f;
         s_q.alpha = ok ? alpha : 0.0f;
         s_q.inv_step = p.inv_step;
+        s_q.inv_step_l = scaled_inv_step(p.inv_step, 1u << BITS);
         s_q.top = static_cast<float>((1 << BITS) - 1);
         s_q.inv_2alpha = inv_2alpha;
         uint32_t cells = 0;
@@ -514,6 +603,13 @@ compress_kernel_dev(const void* __restrict__ grad, uint64_t d, uint64_t grad_str
     }
     if constexpr (NONUNIFORM) {
         if (s_q.cells == 0) return;  // left to compress_kernel_dev_fallback
+    }
+    if constexpr (!NONUNIFORM) {
+        if (s_q.inv_step_l == 0.0f) {    // alpha too large for the scaled inverse step
+            compress_block<BITS, kUniformWide, BF16>(s_q, s_grid, s_cell, s_search, grad, d, grad_stride, rk,
+                                                     first_worker + wi, wi, packed, words_stride, words_out);
+            return;
+        }
     }
     compress_block<BITS, NONUNIFORM ? kGrid : kUniform, BF16>(s_q, s_grid, s_cell, s_search, grad, d, grad_stride, rk,
                                                               first_worker + wi, wi, packed, words_stride, words_out);
@@ -647,6 +743,7 @@ static cudaError_t dispatch(const CompressCall& c, const CompressArgs& a, dim3 g
     }
     if (search == kGrid) return c.bf16 ? launch<BITS, kGrid, true>(c, a, grid) : launch<BITS, kGrid, false>(c, a, grid);
     if (search == kBinary) return c.bf16 ? launch<BITS, kBinary, true>(c, a, grid) : launch<BITS, kBinary, false>(c, a, grid);
+    if (search == kUniformWide) return c.bf16 ? launch<BITS, kUniformWide, true>(c, a, grid) : launch<BITS, kUniformWide, false>(c, a, grid);
     return c.bf16 ? launch<BITS, kUniform, true>(c, a, grid) : launch<BITS, kUniform, false>(c, a, grid);
 }
 
@@ -660,6 +757,8 @@ cudaError_t launch_compress(const CompressCall& c) {
         WorkerQ& q = args.q[i];
         q.alpha = p.alpha; q.inv_step = p.inv_step; q.top = static_cast<float>(p.num_levels - 1);
         q.inv_2alpha = 1.0f / (2.0f * p.alpha);
+        q.inv_step_l = scaled_inv_step(p.inv_step, p.num_levels);
+        if (!c.nonuniform && q.inv_step_l == 0.0f) search = kUniformWide;
         q.cells = 0; q.cell_scale = 0.0f;
         for (int k = 0; k < TQ_MAX_LEVELS; ++k) { q.levels[k] = p.levels[k]; q.inv_width[k] = p.inv_width[k]; }
         if (c.nonuniform) {
@@ -668,7 +767,7 @@ cudaError_t launch_compress(const CompressCall& c) {
             if (q.cells == 0 || !std::isfinite(q.inv_2alpha)) search = kBinary;
         }
     }
-    const dim3 grid = compress_grid(c.d, c.n_workers, search != kUniform);
+    const dim3 grid = compress_grid(c.d, c.n_workers, !is_uniform(search));
     switch (c.bits) {
         case 1: return dispatch<1>(c, args, grid, search);
         case 2: return dispatch<2>(c, args, grid, search);

@@ -76,28 +76,6 @@ __device__ __forceinline__ float load1(const void* base, uint64_t j) {
     else return __uint_as_float(static_cast<uint32_t>(__ldg(reinterpret_cast<const unsigned short*>(base) + j)) << 16);
 }
 
-// ---- Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11) -------------------------------------------
-// Ten rounds; each round multiplies counter words 0 and 2 by fixed odd constants, keeps both halves
-// of the 64-bit products and xors the high halves with the remaining counter words and the round
-// key; the key advances by a Weyl sequence between rounds.
-__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                              uint32_t k0, uint32_t k1, uint32_t (&out)[4]) {
-#pragma unroll
-    for (int r = 0; r < 10; ++r) {
-        const uint64_t p0 = static_cast<uint64_t>(0xD2511F53u) * c0;
-        const uint64_t p1 = static_cast<uint64_t>(0xCD9E8D57u) * c2;
-        const uint32_t n0 = static_cast<uint32_t>(p1 >> 32) ^ c1 ^ k0;
-        const uint32_t n2 = static_cast<uint32_t>(p0 >> 32) ^ c3 ^ k1;
-        c1 = static_cast<uint32_t>(p1);
-        c3 = static_cast<uint32_t>(p0);
-        c0 = n0;
-        c2 = n2;
-        k0 += 0x9E3779B9u;
-        k1 += 0xBB67AE85u;
-    }
-    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
-}
-
 // ---- asynchronous copies into shared memory, counted on an mbarrier ----------------------------------
 // Every wait is bounded: after kWaitLimit polls the caller gets `false`, records it and winds down.
 constexpr uint32_t kWaitLimit = 1u << 22;

@@ -66,23 +66,49 @@ struct TailModel {
         const double t = cbrt(outer) * pow(1.0 - k, 2.0 / 3.0) + cbrt(inner) * pow(k, 2.0 / 3.0);
         return t * t * t;
     }
-    // k* = argmin_k Q_B(a, k): scan k = j/64, then 60 golden-section steps between the neighbours of the best j
+    // d/dx of mass_inside: twice the model density
+    TQ_HD double mass_slope(double x) const {
+        if (x <= g_min) return (1.0 - 2.0 * rho) / g_min;
+        return 2.0 * rho * (gamma - 1.0) / g_min * pow(x / g_min, -gamma);
+    }
+    // A quantity with the sign of dQ_B/dk on 0 < k < 1.  With u = mass_inside(k a), w = mass_inside(a) - u and
+    // Q_B^(1/3) = w^(1/3) (1-k)^(2/3) + u^(1/3) k^(2/3), the derivative times the positive factor
+    // 3 w^(2/3) (1-k)^(1/3) u^(2/3) k^(1/3) is
+    //     w^(2/3) (1-k)^(1/3) (u' k + 2 u)  -  u^(2/3) k^(1/3) (u' (1-k) + 2 w),      u' = a * mass_slope(k a).
+    TQ_HD double biscaled_slope_sign(double a, double k) const {
+        const double u = mass_inside(k * a);
+        double w = mass_inside(a) - u;
+        if (w < 0.0) w = 0.0;
+        const double du = a * mass_slope(k * a);
+        const double cw = cbrt(w), cu = cbrt(u);
+        return cw * cw * cbrt(1.0 - k) * (du * k + 2.0 * u) - cu * cu * cbrt(k) * (du * (1.0 - k) + 2.0 * w);
+    }
+    // k* = argmin_k Q_B(a, k) (Appendix).  Q_B(a, 0) = Q_B(a, 1) = Q_U(a), so the minimum is a point where the
+    // slope turns from negative to positive (at the density's jump, k a = g_min, it may do so without
+    // passing through zero).  Every such turn between neighbours of a 128-point grid is closed in on by
+    // bisection of the slope's sign; the turn with the smallest Q_B wins.  No turn: the minimum is an end.
     TQ_HD double biscaled_split(double a) const {
-        int best = 0;
-        double best_q = biscaled_factor(a, 0.0);
-        for (int j = 1; j <= 64; ++j) {
-            const double q = biscaled_factor(a, j / 64.0);
-            if (q < best_q) { best_q = q; best = j; }
+        constexpr int kGrid = 128;
+        double best_k = 0.0, best_q = biscaled_factor(a, 0.0);
+        constexpr double kFirst = 9.094947017729282e-13;                // 2^-40: the grid's first point, in place of 0
+        bool prev_neg = biscaled_slope_sign(a, kFirst) < 0.0;        // slope at the previous grid point was negative
+        for (int j = 1; j <= kGrid; ++j) {
+            const double k = static_cast<double>(j) / kGrid;
+            // at k = 1 the slope's sign is that of approaching the end from inside: treat the end as a turn
+            const bool neg = j < kGrid ? biscaled_slope_sign(a, k) < 0.0 : false;
+            if (prev_neg && !neg) {
+                double lo = j > 1 ? static_cast<double>(j - 1) / kGrid : kFirst, hi = k;      // slope < 0 at lo, >= 0 at hi
+                for (int it = 0; it < 64 && hi - lo > 0.0; ++it) {
+                    const double mid = 0.5 * (lo + hi);
+                    if (mid <= lo || mid >= hi) break;
+                    if (biscaled_slope_sign(a, mid) < 0.0) lo = mid; else hi = mid;
+                }
+                const double kk = 0.5 * (lo + hi), q = biscaled_factor(a, kk);
+                if (q < best_q) { best_q = q; best_k = kk; }
+            }
+            prev_neg = neg;
         }
-        double lo = (best > 0 ? best - 1 : 0) / 64.0, hi = (best < 64 ? best + 1 : 64) / 64.0;
-        const double r = 0.6180339887498949;
-        double x1 = hi - r * (hi - lo), x2 = lo + r * (hi - lo);
-        double f1 = biscaled_factor(a, x1), f2 = biscaled_factor(a, x2);
-        for (int it = 0; it < 60; ++it) {
-            if (f1 <= f2) { hi = x2; x2 = x1; f2 = f1; x1 = hi - r * (hi - lo); f1 = biscaled_factor(a, x1); }
-            else { lo = x1; x1 = x2; f1 = f2; x2 = lo + r * (hi - lo); f2 = biscaled_factor(a, x2); }
-        }
-        return 0.5 * (lo + hi);
+        return best_k;
     }
     TQ_HD double q_of(uint32_t mode, double a) const {
         if (mode == TQ_UNIFORM) return mass_inside(a);

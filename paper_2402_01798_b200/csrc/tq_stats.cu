@@ -61,7 +61,10 @@ stats_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride, fl
     float g_min = g_min_in;
     if constexpr (PASS == kTail) g_min = stats[wi].g_min;     // finished by the moments pass
     const bool tail_on = (PASS != kMoments) && (g_min > 0.0f);
-    const float inv_gmin = tail_on ? __frcp_rn(g_min) : 0.0f;
+    // Tail elements are scaled by inv_gmin before the logarithm and the exact logarithm of inv_gmin * g_min
+    // is taken out again at the end, so inv_gmin only has to keep |g| * inv_gmin inside the normal range
+    // for |g| > g_min.  1 / g_min overflows for a subnormal g_min; such a threshold is scaled by 2^64 first.
+    const float inv_gmin = tail_on ? __frcp_rn(g_min < 7.8886090522101181e-31f ? g_min * 18446744073709551616.0f : g_min) : 0.0f;
 
     double sum_abs = 0.0, sum_sq = 0.0, sum_log2 = 0.0;
     unsigned long long n_tail = 0, n_bad = 0;
@@ -132,7 +135,7 @@ stats_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride, fl
                 sum_abs += av; sum_sq += static_cast<double>(av) * av; max_abs = fmaxf(max_abs, av); n_bad += ok ? 0 : 1;
             }
             if constexpr (PASS != kMoments) {
-                if (tail_on && ok && a > g_min) { sum_log2 += __log2f(a * inv_gmin); n_tail += 1; }
+                if (tail_on && ok && a > g_min) { sum_log2 += log2(static_cast<double>(a) * static_cast<double>(inv_gmin)); n_tail += 1; }
             }
         }
     }
@@ -199,8 +202,8 @@ stats_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride, fl
             if constexpr (PASS == kMoments) { st->n_tail = 0; st->sum_log_tail = 0.0; }
         }
         if constexpr (PASS != kMoments) {
-            // elements were scaled by fl(1/g_min) instead of divided by g_min: remove the exact
-            // logarithm of that factor's error, n * log2(fl(1/g_min) * g_min), then convert to ln
+            // elements were scaled by inv_gmin instead of divided by g_min: remove the exact
+            // logarithm of that factor's error, n * log2(inv_gmin * g_min), then convert to ln
             double corr = 0.0;
             if (tail_on) corr = static_cast<double>(t.n_tail) * log2(static_cast<double>(inv_gmin) * static_cast<double>(g_min));
             st->n_tail = t.n_tail;

@@ -120,8 +120,18 @@ def test_tq_params_agrees_with_oracle(tq, orc, L, mode, gamma, rule):
         assert a.flags == b.flags
         assert math.isclose(a.alpha, b.alpha, rel_tol=3e-7)
         assert math.isclose(a.gamma, b.gamma, rel_tol=3e-7) and math.isclose(a.rho, b.rho, rel_tol=3e-7)
-        assert np.allclose(list(a.levels), list(b.levels), rtol=5e-7, atol=0)
-        assert np.allclose(list(a.inv_width), list(b.inv_width), rtol=2e-6, atol=0)
+        # BiScaled (mode 2): the Appendix gives no procedure for k* = argmin_k Q_B.  The oracle compares values
+        # of Q_B (scan + golden section), which places a flat minimum only to about the square root of Q_B's
+        # evaluation noise, and that noise grows with alpha / g_min (the outer mass is a difference of two
+        # numbers near 1).  The library bisects the sign of dQ_B/dk instead, which agrees with a 60-digit
+        # evaluation of that root to 1e-13.  With the paper's alpha rules the two agree to fp32 rounding;
+        # only with no truncation at all (rule 3, alpha = max|g| far beyond the fixed point) do they part:
+        # up to 8e-7 at alpha / g_min = 700 and 4e-5 at 1.5e5 (measured; the oracle's k* is off by 1.5e-6 there).
+        lev_tol = 5e-7
+        if mode == 2 and rule == 3:
+            lev_tol = 1e-4 if a.alpha / a.g_min > 1e4 else 2e-6
+        assert np.allclose(list(a.levels), list(b.levels), rtol=lev_tol, atol=0)
+        assert np.allclose(list(a.inv_width), list(b.inv_width), rtol=max(2e-6, 4 * lev_tol), atol=0)
         assert math.isclose(a.inv_step, b.inv_step, rel_tol=3e-7)
         lv = np.array(a.levels[:L], dtype=np.float64)
         assert np.all(np.diff(lv) > 0) and lv[0] == -a.alpha and lv[-1] == a.alpha
