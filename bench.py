@@ -2,11 +2,18 @@
 """Benchmark of the truncated-quantization hot path on B200.
 
 A step is one full round over one batch of synthetic heavy-tailed gradients already resident in
-HBM: statistics (two passes: moments, then the tail beyond g_min = mean|g|) -> closed-form
-parameters (the 64-byte records are copied back and designed on the host: one sync per round;
---device-params designs them on the device instead, with no host round trip) -> fused truncate + stochastic round + pack for all N workers -> fused unpack + dequantize +
-average.  Throughput is bytes of gradient input (N * d * elemsize) per
-second of step time.
+HBM: statistics (default: one pass, g_min = mean|g| rounded down to a power of two, hinted by the
+previous round's mean; --stats two-pass: moments, then the tail beyond g_min = mean|g|) ->
+closed-form parameters (the 64-byte records are copied back and designed on the host: one sync per
+round; --device-params designs them on the device instead, with no host round trip) -> fused
+truncate + stochastic round + pack for all N workers -> fused unpack + dequantize + average.
+Throughput is bytes of gradient input (N * d * elemsize) per second of step time.
+
+The headline numbers (value, roofline, e2e, cpu_baseline) are those of --config (default: 25.6 M x 16
+fp32).  On one GPU the line also carries, under "workloads", the per-kernel times (median, min, mean),
+algorithmic bytes, fraction of the measured copy peak and sampled clocks of the other workloads with
+d >= 25.6 M: 124 M x 8 stored as bf16 (uniform and non-uniform, 4 and 16 levels) and 10^9 x 4; each is
+generated, timed and freed in turn (--no-workloads leaves them out).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config 0..4] [--impl ours|reference]
 
@@ -48,7 +55,7 @@ def hbm_peak():
 class ClockSampler:
     """Samples SM clocks and throttle reasons through NVML (read-only) while the timed region runs."""
 
-    def __init__(self, index: int, period_s: float = 0.01):
+    def __init__(self, index: int, period_s: float = 0.001):
         self.index, self.period, self.samples, self.reasons = index, period_s, [], set()
         self.max_mhz, self.stop_flag, self.thread, self.err = None, False, None, None
 
@@ -267,61 +274,17 @@ def run_exchange(args, w, tq, rank, local_rank, world, dev):
     dist.destroy_process_group()
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
-    ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--config", type=int, default=2, help="index into the five workloads (default: 25.6M x 16)")
-    ap.add_argument("--variant", type=int, default=None,
-                    help="with --config 3: index 0..11 into the bf16 sweep (gamma x mode x levels)")
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--device-params", action="store_true",
-                    help="design the parameters on the device (tq_params_device): no host round trip inside the round")
-    ap.add_argument("--stats", default="hinted", choices=["two-pass", "hinted"],
-                    help="two-pass: g_min = mean|g| (tq_stats); hinted: g_min = mean|g| rounded down to a power of two, "
-                         "one pass over the data with the previous round's mean as the hint (tq_stats_hinted)")
-    ap.add_argument("--exchange", default="replicas", choices=["replicas", "allgather", "peer"],
-                    help="replicas (default): every rank runs its own copy of the workload, nothing crosses ranks; "
-                         "allgather: the N workers are split over the ranks and the packed rows are all-gathered (NCCL) "
-                         "before the aggregation; peer: same split, the aggregation kernel reads the peers' rows in place")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-e2e", action="store_true")
-    args = ap.parse_args()
-    args.host_params = not args.device_params
-    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-
-    from paper_2402_01798_b200 import inputs
-    w = inputs.WORKLOADS[args.config]
-    if args.config == 3 and args.variant is not None:
-        w = inputs.CONFIG4_SWEEP[args.variant]
-    if args.impl == "reference":
-        run_reference(args, w)
-        return
-
+def measure_round(args, tq, w, g, stride, dev, local_rank, world, steps, warmup, headline):
+    """Times `steps` rounds of workload `w` on the gradients `g` already resident in HBM (CUDA events on the
+    launching stream, clocks sampled meanwhile).  headline=True adds the roofline object, the end-to-end
+    measurement with host buffers and the CPU oracle beside it."""
     import torch
-    from paper_2402_01798_b200 import binding as tq
-
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    tq.lib()
-    if args.exchange != "replicas":
-        run_exchange(args, w, tq, rank, local_rank, world, dev)
-        return
-
     esz = 2 if w.dtype == torch.bfloat16 else 4
     mode = tq.NONUNIFORM if w.mode == "nonuniform" else tq.UNIFORM
     N, d, bits = w.n_workers, w.d, w.bits
 
-    # inputs resident in HBM (rank r uses its own seeds: a replica, not a shard)
-    wr = replica_workload(w, rank)
-    g, stride = inputs.make_worker_gradients(wr, dev)
+    rank = int(os.environ.get("RANK", "0"))
+    stats_t = lambda xs: {"ms": statistics.mean(xs), "ms_median": statistics.median(xs), "ms_min": min(xs)}
     words = tq.tq_packed_words(d, bits)
     packed = torch.empty((N, words), dtype=torch.int32, device=dev)
     out = torch.empty(d, dtype=torch.float32, device=dev)
@@ -368,18 +331,18 @@ def main():
             torch.distributed.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
+    for _ in range(warmup):
         one_round()
     barrier()
 
     sampler = ClockSampler(local_rank)
     sampler.start()
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(steps)]
     l0 = tq.tq_kernel_launches()
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     t_start.record()
-    for k in range(args.steps):
+    for k in range(steps):
         one_round(evs[k])
     t_end.record()
     barrier()
@@ -388,15 +351,15 @@ def main():
     total_ms = t_start.elapsed_time(t_end)
 
     total_ms = max_over_ranks(total_ms, world, dev)
-    ms_per_step = total_ms / args.steps
+    ms_per_step = total_ms / steps
     in_bytes = N * d * esz
     value = whole_job_gbs(world, in_bytes, ms_per_step)
 
     # per-kernel durations inside the timed region (CUDA events on the launching stream)
-    t_stats = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)       # two launches
-    t_params = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)      # device kernel, or copy + sync + host design
-    t_comp = statistics.mean(e[2].elapsed_time(e[3]) for e in evs)
-    t_dec = statistics.mean(e[3].elapsed_time(e[4]) for e in evs)
+    t_stats = stats_t([e[0].elapsed_time(e[1]) for e in evs])       # two launches
+    t_params = stats_t([e[1].elapsed_time(e[2]) for e in evs])      # device kernel, or copy + sync + host design
+    t_comp = stats_t([e[2].elapsed_time(e[3]) for e in evs])
+    t_dec = stats_t([e[3].elapsed_time(e[4]) for e in evs])
     peak, peak_kind = hbm_peak()
     stats_passes = 1 if args.stats == "hinted" else 2     # hinted: the second kernel returns at once when the hint holds
     stats_key = "tq_stats (hinted, 1 pass)" if args.stats == "hinted" else "tq_stats (2 passes)"
@@ -405,10 +368,16 @@ def main():
         "tq_compress": (N * d * esz + N * d * bits // 8, t_comp, 1),
         "tq_decompress_aggregate": (N * d * bits // 8 + 4 * d, t_dec, 1),
     }
-    kernels = {"tq_params": {"ms": t_params, "where": "host (one sync)" if args.host_params else "device kernel"}}
-    kernels.update({k: {"ms": t, "launches_per_step": n, "algorithmic_bytes": b, "gbs": b / (t * 1e-3) / 1e9,
-                   "frac_of_hbm_peak": b / (t * 1e-3) / 1e9 / peak} for k, (b, t, n) in alg.items()})
+    kernels = {"tq_params": dict(t_params, where="host (one sync)" if args.host_params else "device kernel")}
+    # gbs / frac_of_hbm_peak from the mean over the timed steps; *_best from the fastest step
+    kernels.update({k: dict(t, launches_per_step=n, algorithmic_bytes=b, gbs=b / (t["ms"] * 1e-3) / 1e9,
+                            frac_of_hbm_peak=b / (t["ms"] * 1e-3) / 1e9 / peak,
+                            frac_of_hbm_peak_median=b / (t["ms_median"] * 1e-3) / 1e9 / peak,
+                            frac_of_hbm_peak_best=b / (t["ms_min"] * 1e-3) / 1e9 / peak) for k, (b, t, n) in alg.items()})
 
+    result = {"ms_per_step": ms_per_step, "value": value, "kernels": kernels, "clocks": clocks, "launches": int(launches),
+              "whole_round_frac": (sum(b for b, _, _ in alg.values()) / (ms_per_step * 1e-3) / 1e9) / peak,
+              "roofline": None, "cpu": None, "e2e": None}
     if args.stats == "hinted":
         # what the statistics cost when the hint does not hold (first round, or the mean moved to another binade):
         # the tail kernel then reads the data a second time
@@ -420,6 +389,7 @@ def main():
             torch.cuda.synchronize()
             miss.append(a.elapsed_time(b))
         kernels[stats_key]["hint_miss_ms"] = statistics.mean(miss)
+        result["round_ms_hint_miss"] = ms_per_step + statistics.mean(miss) - t_stats["ms"]
         run_stats(g)                                     # leave a valid hint behind
 
     # decompress-aggregate again with the packed rows evicted from L2 first (in the round above they
@@ -436,14 +406,18 @@ def main():
     t_cold = statistics.mean(cold)
     kb = alg["tq_decompress_aggregate"][0]
     kernels["tq_decompress_aggregate"]["cold_l2_ms"] = t_cold
+    kernels["tq_decompress_aggregate"]["cold_l2_ms_min"] = min(cold)
     kernels["tq_decompress_aggregate"]["cold_l2_gbs"] = kb / (t_cold * 1e-3) / 1e9
     kernels["tq_decompress_aggregate"]["cold_l2_frac_of_hbm_peak"] = kb / (t_cold * 1e-3) / 1e9 / peak
     del flush
+    result["checksum"] = float(out.double().sum().item())
+    if not headline:
+        return result
 
     dom = "tq_compress"      # the single kernel with the largest share of the round (see profiles/launch_list_*)
-    roofline = {"kernel": dom, "bound": "hbm", "achieved": kernels[dom]["gbs"], "peak": peak, "peak_source": peak_kind,
-                "unit": "GB/s", "frac": kernels[dom]["gbs"] / peak, "algorithmic_bytes": alg[dom][0],
-                "traffic": NCU_DRAM_BYTES.get((w.name, dom))}
+    result["roofline"] = {"kernel": dom, "bound": "hbm", "achieved": kernels[dom]["gbs"], "peak": peak, "peak_source": peak_kind,
+                          "unit": "GB/s", "frac": kernels[dom]["gbs"] / peak, "algorithmic_bytes": alg[dom][0],
+                          "traffic": NCU_DRAM_BYTES.get((w.name, dom))}
 
     # end to end through the public API with HOST buffers: H2D of every worker's gradient, the round,
     # D2H of the aggregated update, all inside the timed region
@@ -456,7 +430,7 @@ def main():
         # returns its result (every step still copies its own inputs in and its own result out)
         bufs = [torch.empty_like(g), torch.empty_like(g)]
         copy_stream = torch.cuda.Stream(device=dev)
-        e2e_steps = max(2, min(args.steps, 5))
+        e2e_steps = max(2, min(steps, 5))
 
         def e2e_compute(g2):
             run_stats(g2)
@@ -500,9 +474,10 @@ def main():
         barrier()
         ems = a.elapsed_time(b)
         ems = max_over_ranks(ems, world, dev) / e2e_steps
-        e2e = {"value": whole_job_gbs(world, in_bytes, ems), "unit": "GB/s", "ms_per_step": ems,
+        e2e = {"value": whole_job_gbs(world, in_bytes, ems), "unit": "GB/s", "ms_per_step": ems, "steps": e2e_steps,
                "h2d_bytes_per_step": int(N * stride * esz), "d2h_bytes_per_step": int(4 * d + 64 * N)}
         del host_g, host_out, bufs
+    result["e2e"] = e2e
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -511,26 +486,110 @@ def main():
         cpu = {"value": N * sample_d * esz / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle", "seconds": dt,
                "host_cores_available": os.cpu_count(),
                "sample": f"{N} workers x {sample_d} elements of workload {w.name}, one full round"}
+    result["cpu"] = cpu
+    return result
+
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=2, help="index into the five workloads (default: 25.6M x 16)")
+    ap.add_argument("--variant", type=int, default=None,
+                    help="with --config 3: index 0..11 into the bf16 sweep (gamma x mode x levels)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--device-params", action="store_true",
+                    help="design the parameters on the device (tq_params_device): no host round trip inside the round")
+    ap.add_argument("--stats", default="hinted", choices=["two-pass", "hinted"],
+                    help="two-pass: g_min = mean|g| (tq_stats); hinted: g_min = mean|g| rounded down to a power of two, "
+                         "one pass over the data with the previous round's mean as the hint (tq_stats_hinted)")
+    ap.add_argument("--exchange", default="replicas", choices=["replicas", "allgather", "peer"],
+                    help="replicas (default): every rank runs its own copy of the workload, nothing crosses ranks; "
+                         "allgather: the N workers are split over the ranks and the packed rows are all-gathered (NCCL) "
+                         "before the aggregation; peer: same split, the aggregation kernel reads the peers' rows in place")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-workloads", action="store_true",
+                    help="leave out the per-kernel measurements of the other d >= 25.6 M workloads")
+    args = ap.parse_args()
+    args.host_params = not args.device_params
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    from paper_2402_01798_b200 import inputs
+    w = inputs.WORKLOADS[args.config]
+    if args.config == 3 and args.variant is not None:
+        w = inputs.CONFIG4_SWEEP[args.variant]
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    from paper_2402_01798_b200 import binding as tq
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    tq.lib()
+    if args.exchange != "replicas":
+        run_exchange(args, w, tq, rank, local_rank, world, dev)
+        return
+
+    wr = replica_workload(w, rank)                      # rank r uses its own seeds: a replica, not a shard
+    g, stride = inputs.make_worker_gradients(wr, dev)
+    head = measure_round(args, tq, wr, g, stride, dev, local_rank, world, args.steps, args.warmup, headline=True)
+    del g
+
+    # the other workloads with d >= 25.6 M (one GPU only: they would hold every rank for a while longer)
+    workloads = None
+    if world == 1 and not args.no_workloads:
+        workloads = {}
+        c4 = {(c.gamma, c.mode, c.num_levels): c for c in inputs.CONFIG4_SWEEP}
+        groups = [[(inputs.WORKLOADS[2], 100)],
+                  [(c4[(3.0, m, L)], 40) for m in ("nonuniform", "uniform") for L in (16, 4)],    # one set of gradients, four quantizers
+                  [(inputs.WORKLOADS[4], 12)]]
+        groups = [[(w2, k) for w2, k in grp if w2.name != w.name] for grp in groups]
+        for group in (grp for grp in groups if grp):
+            torch.cuda.empty_cache()
+            g2, stride2 = inputs.make_worker_gradients(group[0][0], dev)
+            for w2, steps2 in group:                    # same gradient data, different quantizers
+                r = measure_round(args, tq, w2, g2, stride2, dev, local_rank, 1, steps2, 3, headline=False)
+                workloads[w2.name] = {"d": w2.d, "n_workers": w2.n_workers, "mode": w2.mode, "levels": w2.num_levels,
+                                      "storage": str(w2.dtype).split(".")[-1], "steps": steps2, "ms_per_step": r["ms_per_step"],
+                                      "value_gbs": r["value"], "hbm_frac_of_peak_whole_round": r["whole_round_frac"],
+                                      "kernels": r["kernels"], "clocks": r["clocks"]}
+            del g2
 
     if rank == 0:
+        d, N, bits = w.d, w.n_workers, w.bits
+        words = tq.tq_packed_words(d, bits)
+        in_bytes = N * d * (2 if w.dtype == torch.bfloat16 else 4)
         line = {
-            "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "metric": METRIC, "value": head["value"], "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "d": d, "n_workers": N, "mode": w.mode, "levels": w.num_levels, "bits": bits,
                        "gamma": w.gamma, "scale": w.scale, "storage": str(w.dtype).split(".")[-1],
                        "g_min": ("mean|g| per worker rounded down to a power of two; one statistics pass, hinted by the previous round's mean "
-                                 "(same data every round, so the hint always holds; when it does not, the tail pass runs again: --stats two-pass "
-                                 "shows that cost)" if args.stats == "hinted"
+                                 "(same data every round, so the hint always holds; when it does not, the tail pass runs again: "
+                                 "kernels[...].hint_miss_ms and round_ms_hint_miss show that cost)" if args.stats == "hinted"
                                  else "mean|g| per worker (two statistics passes)"), "alpha_rule": "fixed point",
                        "params": "host" if args.host_params else "device (no host round trip inside the round)",
                        "l2": f"inputs ({in_bytes / 1e6:.0f} MB) exceed L2; packed rows ({N * words * 4 / 1e6:.0f} MB) are "
                              "re-read right after being written, see kernels.tq_decompress_aggregate.cold_l2_*",
                        "multi_gpu": "independent replica per rank, no data-path collective"},
-            "hbm_frac_of_peak_whole_round": (sum(b for b, _, _ in alg.values()) / (ms_per_step * 1e-3) / 1e9) / peak,
-            "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu, "e2e": e2e,
-            "gpu_launches": int(launches), "clocks": clocks,
-            "update_checksum": float(out.double().sum().item()),      # rank 0's aggregated update, for comparing variants
+            "hbm_frac_of_peak_whole_round": head["whole_round_frac"],
+            "round_ms_hint_miss": head.get("round_ms_hint_miss"),
+            "roofline": head["roofline"], "kernels": head["kernels"], "cpu_baseline": head["cpu"], "e2e": head["e2e"],
+            "gpu_launches": head["launches"], "clocks": head["clocks"],
+            "update_checksum": head["checksum"],      # rank 0's aggregated update, for comparing variants
+            "workloads": workloads,
         }
         print(json.dumps(line), flush=True)
     if world > 1:

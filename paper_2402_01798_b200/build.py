@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libtq.so")
-SOURCES = ["tq_api.cu", "tq_stats.cu", "tq_compress.cu", "tq_decompress.cu", "tq_params.cu"]
+SOURCES = ["tq_api.cu", "tq_stats.cu", "tq_compress.cu", "tq_compress_lut.cu", "tq_decompress.cu", "tq_params.cu"]
 HEADERS = ["tq_device.cuh", "tq_launch.h"]
 
 NVCC_FLAGS = [

@@ -87,26 +87,38 @@ __device__ __forceinline__ float rounds_up(float p, float rf) {
 //   y   = sat(sum * (inv_step / L))            = clip(x, 0, L) / L exactly: scaling by a power of two commutes
 //                                                with the rounding of the product, and .sat sends NaN and
 //                                                negatives to 0, which is where the reference sends them
-//   y  -= sat(y - s/L)                         = min(y, s/L): for y in (s/L, 1] the difference is exact
-//                                                (s/L >= 1/2, Sterbenz), so the result is s/L itself; this is
-//                                                x = s, which the reference codes as s, like every g >= alpha
+//   y   = min(y, s/L)                          this is x = s, which the reference codes as s, like every g >= alpha
 //   Xm  = fma(y, L * 2^16, 2^23)               = 2^23 + X, rounded to nearest-even as rint does (2^23 is even)
 //   v   = Xm - (2^23 + r)                      = X - r, exact
 //   cm  = fma.rp(v, 2^-16, 1.5 * 2^23)         = 1.5 * 2^23 + ceil(v / 2^16): the sum stays inside one binade
-// and the caller subtracts the bias (or most of it, see pack8).  sum0 / sum1 are g + alpha of the pair.
+// and the caller subtracts the bias.  sum0 / sum1 are g + alpha of the pair.
 struct UniformQ {
     float inv_step_l, c_top;      // inv_step / L, s / L
     f32x2 scale2;                 // L * 2^16, twice
+    f32x2 scale2_dn;              // L * 2^16 * 2^-100, twice (codes as denormals, see code_uniform2_dn)
 };
 constexpr float kCodeBias = 12582912.0f;                 // 1.5 * 2^23
 __device__ __forceinline__ f32x2 fma2_ru(f32x2 a, f32x2 b, f32x2 c) {   // round toward +infinity
     f32x2 r; asm("fma.rp.f32x2 %0, %1, %2, %3;" : "=l"(r.v) : "l"(a.v), "l"(b.v), "l"(c.v)); return r;
 }
+__device__ __forceinline__ f32x2 mul2_ru(f32x2 a, f32x2 b) {
+    f32x2 r; asm("mul.rp.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v)); return r;
+}
+// min(y, s/L) runs on the integer/compare pipe, which has room here; the multiply-add pipes do not.
 __device__ __forceinline__ f32x2 code_uniform2(float sum0, float sum1, const UniformQ& u, float rf0, float rf1) {
-    const float y0 = mul_sat(sum0, u.inv_step_l), y1 = mul_sat(sum1, u.inv_step_l);
-    const f32x2 y = sub2(pair(y0, y1), pair(sub_sat(y0, u.c_top), sub_sat(y1, u.c_top)));
+    const f32x2 y = pair(fminf(mul_sat(sum0, u.inv_step_l), u.c_top), fminf(mul_sat(sum1, u.inv_step_l), u.c_top));
     const f32x2 v = sub2(fma2(y, u.scale2, both(kMagic)), pair(rf0, rf1));
     return fma2_ru(v, both(1.52587890625e-5f), both(kCodeBias));
+}
+// The same with everything scaled by 2^-100: Xm = fma(y, L * 2^16 * 2^-100, 2^-77) = 2^-77 + X * 2^-100 (rounded
+// at 2^-100 exactly as the unscaled form rounds at 1), the slot arrives as 2^-77 + r * 2^-100, and
+// (X - r) * 2^-100 * 2^-65 rounded up is ceil((X - r) / 2^16) * 2^-149: a denormal whose bit pattern is the code
+// itself, with no bias to take off (or -0 when X < r: pack8_bits' callers drop the sign bit).
+constexpr uint32_t kSlotExpBits = 0x19000000u;            // 2^-77
+__device__ __forceinline__ f32x2 code_uniform2_dn(float sum0, float sum1, const UniformQ& u, float rf0, float rf1) {
+    const f32x2 y = pair(fminf(mul_sat(sum0, u.inv_step_l), u.c_top), fminf(mul_sat(sum1, u.inv_step_l), u.c_top));
+    const f32x2 v = sub2(fma2(y, u.scale2_dn, both(6.617444900424222e-24f)), pair(rf0, rf1));
+    return mul2_ru(v, both(2.710505431213761e-20f));     // 2^-65
 }
 
 // The same decision without the scaled inverse step (alpha so large that inv_step / L is subnormal):
@@ -179,68 +191,33 @@ __device__ __forceinline__ float code_binary(float g, float alpha, const float* 
 
 // Four pairs of float codes (elements 0..7 of a group, each code < 2^BITS) -> their 8*BITS packed
 // bits, LSB first.  Every partial sum is an integer below 2^24, so the fp32 arithmetic is exact.
-// Returns a word whose low 8*BITS bits are the packed codes; with BIASED (2- and 4-bit codes only) the
-// bits above them are not zero and the caller merges chunks by byte-permutes.
+// Returns a word whose low 8*BITS bits are the packed codes.
 //
-// BIASED: the caller left 2^23 in the even element of pair 0 (and of pair 2 for 4-bit codes), see
-// code_bias().  The 16-bit partial results then appear as 2^23 + value, whose bit pattern holds the
-// value in its low half, and no float -> integer conversion is needed.
-template <int BITS, bool BIASED>
+// DN (2- and 4-bit codes only): the codes are denormals whose bit pattern is the code (see
+// code_uniform2_dn), sums and products of them are fixed-point arithmetic in units of 2^-149, and the
+// packed bits appear as a bit pattern without any float -> integer conversion.  Bits above the low 16 of
+// a partial result may be set (a sum of -0 terms is -0): the caller merges chunks by byte-permutes that
+// take the low 16 bits only.
+template <int BITS, bool DN>
 __device__ __forceinline__ uint32_t pack8(const f32x2 (&c)[4]) {
     constexpr float B = static_cast<float>(1 << BITS), B2 = B * B;
-    static_assert(!BIASED || BITS == 2 || BITS == 4, "only 16-bit partial results fit beside the bias");
+    static_assert(!DN || BITS == 2 || BITS == 4, "the callers of the denormal form keep 16 bits of each partial result");
     if constexpr (BITS <= 3) {
         f32x2 a = fma2(c[3], both(B2), c[2]);
         a = fma2(a, both(B2), c[1]);
         a = fma2(a, both(B2), c[0]);
         float ev, od;
         unpair(a, ev, od);
-        if constexpr (BIASED) return __float_as_uint(__fmaf_rn(od, B, ev));   // 2^23 + 16 bits
+        if constexpr (DN) return __float_as_uint(__fmaf_rn(od, B, ev));
         else return __float2uint_rz(__fmaf_rn(od, B, ev));
     } else {
         float e0, o0, e1, o1;
         unpair(fma2(c[1], both(B2), c[0]), e0, o0);       // elements 0..3: 16 bits
         unpair(fma2(c[3], both(B2), c[2]), e1, o1);       // elements 4..7: 16 bits
-        if constexpr (BIASED)
+        if constexpr (DN)
             return __byte_perm(__float_as_uint(__fmaf_rn(o0, B, e0)), __float_as_uint(__fmaf_rn(o1, B, e1)), 0x5410u);
         else return __float2uint_rz(__fmaf_rn(o0, B, e0)) + (__float2uint_rz(__fmaf_rn(o1, B, e1)) << 16);
     }
-}
-// What to subtract from code_uniform2's result for pair h of a group so that pack8<BITS, BIASED> can
-// take it: the whole bias 1.5 * 2^23, except 2^22 in the even element of the pairs that start a 16-bit
-// partial result, which therefore keeps 2^23.
-template <int BITS, bool BIASED>
-__device__ __forceinline__ f32x2 code_bias(int h) {
-    const bool keep = BIASED && (h == 0 || (BITS == 4 && h == 2));
-    return pair(keep ? 4194304.0f : kCodeBias, kCodeBias);
-}
-
-// The ten Philox round keys (key advanced by the Weyl constants), computed once on the host: they
-// depend on the seed only, and sit in the kernel's constant bank instead of registers.
-struct RoundKeys {
-    uint32_t k0[10], k1[10];
-};
-
-__device__ __forceinline__ void mul_wide(uint32_t a, uint32_t b, uint32_t& hi, uint32_t& lo) {
-    uint64_t p;
-    asm("mul.wide.u32 %0, %1, %2;" : "=l"(p) : "r"(a), "r"(b));
-    asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(p));
-}
-
-// Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11) with the key schedule supplied.
-__device__ __forceinline__ void philox_rounds(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                              const RoundKeys& rk, uint32_t (&out)[4]) {
-#pragma unroll
-    for (int r = 0; r < 10; ++r) {
-        uint32_t hi0, lo0, hi1, lo1;
-        mul_wide(0xD2511F53u, c0, hi0, lo0);
-        mul_wide(0xCD9E8D57u, c2, hi1, lo1);
-        c0 = hi1 ^ c1 ^ rk.k0[r];
-        c2 = hi0 ^ c3 ^ rk.k1[r];
-        c1 = lo1;
-        c3 = lo0;
-    }
-    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
 struct RunCtx {
@@ -252,7 +229,7 @@ struct RunCtx {
 template <int BITS>
 __device__ __forceinline__ UniformQ uniform_q(const WorkerQ& q) {
     constexpr float L = static_cast<float>(1 << BITS);
-    return UniformQ{q.inv_step_l, (L - 1.0f) / L, both(L * 65536.0f)};
+    return UniformQ{q.inv_step_l, (L - 1.0f) / L, both(L * 65536.0f), both(L * 65536.0f * 7.888609052210118e-31f)};
 }
 
 // inv_step / L for the scaled uniform path: exact when the quotient is a normal number (L is a power of
@@ -262,9 +239,10 @@ __host__ __device__ inline float scaled_inv_step(float inv_step, uint32_t num_le
     return (q >= 1.17549435e-38f && q <= 3.402823466e38f) ? q : 0.0f;
 }
 
-// the 16 random bits of slot e of a Philox block, as the float 2^23 + r
+// the 16 random bits of slot e of a Philox block, as the float 2^23 + r (DN: 2^-77 + r * 2^-100)
+template <bool DN>
 __device__ __forceinline__ float slot_as_float(const uint32_t (&rnd)[4], int e) {
-    return __uint_as_float(__byte_perm(rnd[e >> 1], kMagicBits, (e & 1) ? 0x7432u : 0x7410u));
+    return __uint_as_float(__byte_perm(rnd[e >> 1], DN ? kSlotExpBits : kMagicBits, (e & 1) ? 0x7432u : 0x7410u));
 }
 
 template <int BITS, int SEARCH, bool BF16, bool TAIL>
@@ -300,24 +278,26 @@ template <int BITS, int SEARCH, bool BF16, bool TAIL>
 __device__ __forceinline__ void quantize_run(const Raw8<BF16> (&g)[4], uint32_t* prow, uint64_t run, uint64_t d, uint64_t words_out,
                                              uint32_t worker, const RoundKeys& rk, const RunCtx& cx) {
     const uint64_t j0 = run << 5;
-    const uint32_t blk_lo = static_cast<uint32_t>(j0 >> 3), blk_hi = static_cast<uint32_t>(j0 >> 35);
+    const uint32_t blk_lo = static_cast<uint32_t>(j0 >> 3);
+    const PhiloxRun pr = philox_run(static_cast<uint32_t>(j0 >> 35), worker, rk);
     const f32x2 alpha2 = both(cx.alpha), inv_step2 = both(cx.inv_step), cell_scale2 = both(cx.cell_scale);
-    // whole runs of the scaled uniform path hand pack8 biased codes (2- and 4-bit codes)
-    constexpr bool BIASED = SEARCH == kUniform && !TAIL && (BITS == 2 || BITS == 4);
+    // whole runs of the scaled uniform path hand pack8 the codes as denormals (2- and 4-bit codes)
+    constexpr bool DN = SEARCH == kUniform && !TAIL && (BITS == 2 || BITS == 4);
     uint32_t chunk[4];   // the 8*BITS packed bits of each group
 #pragma unroll
     for (int grp = 0; grp < 4; ++grp) {
         uint32_t rnd[4];
-        philox_rounds(blk_lo + grp, blk_hi, worker, 0u, rk, rnd);     // j0 >> 3 is a multiple of 4: no carry
+        philox_block(blk_lo + grp, pr, rk, rnd);                      // j0 >> 3 is a multiple of 4: no carry
         f32x2 code[4];
 #pragma unroll
         for (int h = 0; h < 4; ++h) {            // elements 2h, 2h+1 of the group
             const int e = 2 * h;
-            const float rf0 = slot_as_float(rnd, e), rf1 = slot_as_float(rnd, e + 1);
+            const float rf0 = slot_as_float<DN>(rnd, e), rf1 = slot_as_float<DN>(rnd, e + 1);
             if constexpr (is_uniform(SEARCH)) {
                 float sum0, sum1;
                 pair_plus_alpha<BF16>(g[grp], h, cx.alpha, sum0, sum1);
-                if constexpr (SEARCH == kUniform) code[h] = sub2(code_uniform2(sum0, sum1, cx.u, rf0, rf1), code_bias<BITS, BIASED>(h));
+                if constexpr (DN) code[h] = code_uniform2_dn(sum0, sum1, cx.u, rf0, rf1);
+                else if constexpr (SEARCH == kUniform) code[h] = sub2(code_uniform2(sum0, sum1, cx.u, rf0, rf1), both(kCodeBias));
                 else code[h] = code_uniform2_wide(sum0, sum1, inv_step2, cx.top, rf0, rf1);
             } else {
                 const float g0 = elem<BF16>(g[grp], e), g1 = elem<BF16>(g[grp], e + 1);
@@ -334,7 +314,7 @@ __device__ __forceinline__ void quantize_run(const Raw8<BF16> (&g)[4], uint32_t*
                 code[h] = pair(c0, c1);
             }
         }
-        chunk[grp] = pack8<BITS, BIASED>(code);
+        chunk[grp] = pack8<BITS, DN>(code);
     }
 
     // four chunks of 8*BITS bits -> BITS words, LSB first
@@ -653,13 +633,6 @@ static uint32_t choose_cells(const tq_params_t& p, float inv_2alpha) {
     return 0;
 }
 
-static RoundKeys round_keys(uint64_t seed) {
-    RoundKeys rk;
-    uint32_t k0 = static_cast<uint32_t>(seed), k1 = static_cast<uint32_t>(seed >> 32);
-    for (int r = 0; r < 10; ++r) { rk.k0[r] = k0; rk.k1[r] = k1; k0 += 0x9E3779B9u; k1 += 0xBB67AE85u; }
-    return rk;
-}
-
 // Persistent grid: 4 resident blocks per SM spread over the workers (table modes build their lookup
 // grid once per block); uniform mode has no per-block set-up, so one block per tile lets the hardware
 // scheduler balance the tail.
@@ -750,6 +723,11 @@ static cudaError_t dispatch(const CompressCall& c, const CompressArgs& a, dim3 g
 cudaError_t launch_compress(const CompressCall& c) {
     if (c.d == 0) return cudaSuccess;
     if (c.params_dev) return launch_compress_dev(c);
+    {
+        bool applied = false;
+        const cudaError_t e = launch_compress_lut(c, &applied);
+        if (applied || e != cudaSuccess) return e;
+    }
     static thread_local CompressArgs args;   // 9 KB: keep it off the stack
     int search = c.nonuniform ? kGrid : kUniform;
     for (uint32_t i = 0; i < c.n_workers; ++i) {

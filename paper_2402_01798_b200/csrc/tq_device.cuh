@@ -134,6 +134,62 @@ __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
     f32x2 r; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r.v) : "l"(a.v), "l"(b.v), "l"(c.v)); return r;
 }
 
+// ---- Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11), counter = (c0, c1, worker, 0) ------------------
+// The ten round keys (key advanced by the Weyl constants) are computed once on the host: they depend on
+// the seed only, and sit in the kernel's constant bank instead of registers.
+struct RoundKeys {
+    uint32_t k0[10], k1[10];
+};
+inline RoundKeys round_keys(uint64_t seed) {
+    RoundKeys rk;
+    uint32_t k0 = static_cast<uint32_t>(seed), k1 = static_cast<uint32_t>(seed >> 32);
+    for (int r = 0; r < 10; ++r) { rk.k0[r] = k0; rk.k1[r] = k1; k0 += 0x9E3779B9u; k1 += 0xBB67AE85u; }
+    return rk;
+}
+
+__device__ __forceinline__ void mul_wide(uint32_t a, uint32_t b, uint32_t& hi, uint32_t& lo) {
+    uint64_t p;
+    asm("mul.wide.u32 %0, %1, %2;" : "=l"(p) : "r"(a), "r"(b));
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(p));
+}
+
+// Within a run of elements only c0 changes, so what the first two rounds make of the other three counter
+// words is computed once per run: of the 20 wide multiplies of a block, 3 drop out (the second product of
+// round 1 and the first of round 2 have constant operands, and word 0 after round 1 is constant).
+struct PhiloxRun {
+    uint32_t a1, b1, b2, d2;
+};
+__device__ __forceinline__ PhiloxRun philox_run(uint32_t c1, uint32_t worker, const RoundKeys& rk) {
+    uint32_t hi1, lo1;
+    mul_wide(0xCD9E8D57u, worker, hi1, lo1);                  // round 1, second product
+    const uint32_t c0_1 = hi1 ^ c1 ^ rk.k0[0];                // word 0 after round 1
+    uint32_t hi0c, lo0c;
+    mul_wide(0xD2511F53u, c0_1, hi0c, lo0c);                  // round 2, first product
+    PhiloxRun r;
+    r.a1 = rk.k1[0];                 // word 2 after round 1 = hi(M0 * c0) ^ 0 ^ k1[0]
+    r.b1 = lo1 ^ rk.k0[1];           // word 0 after round 2 = hi(M1 * word 2) ^ lo1 ^ k0[1]
+    r.b2 = hi0c ^ rk.k1[1];          // word 2 after round 2 = hi0c ^ lo(M0 * c0) ^ k1[1]
+    r.d2 = lo0c;                     // word 3 after round 2
+    return r;
+}
+__device__ __forceinline__ void philox_block(uint32_t c0, const PhiloxRun& pr, const RoundKeys& rk, uint32_t (&out)[4]) {
+    uint32_t hi0, lo0, hi1, lo1;
+    mul_wide(0xD2511F53u, c0, hi0, lo0);                      // round 1
+    const uint32_t w2 = hi0 ^ pr.a1;
+    mul_wide(0xCD9E8D57u, w2, hi1, lo1);                      // round 2
+    uint32_t x0 = hi1 ^ pr.b1, x1 = lo1, x2 = lo0 ^ pr.b2, x3 = pr.d2;
+#pragma unroll
+    for (int r = 2; r < 10; ++r) {
+        mul_wide(0xD2511F53u, x0, hi0, lo0);
+        mul_wide(0xCD9E8D57u, x2, hi1, lo1);
+        x0 = hi1 ^ x1 ^ rk.k0[r];
+        x2 = hi0 ^ x3 ^ rk.k1[r];
+        x1 = lo1;
+        x3 = lo0;
+    }
+    out[0] = x0; out[1] = x1; out[2] = x2; out[3] = x3;
+}
+
 // ---- warp / block reductions -----------------------------------------------------------------------
 __device__ __forceinline__ double warp_sum(double v) {
 #pragma unroll

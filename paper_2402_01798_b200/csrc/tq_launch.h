@@ -17,6 +17,9 @@ struct CompressCall {
     cudaStream_t stream;
 };
 cudaError_t launch_compress(const CompressCall& c);
+// bf16 rows through the per-bit-pattern decision table; *applied is false (and nothing is launched) when the
+// table form does not fit the call, which then takes the element-wise kernels.
+cudaError_t launch_compress_lut(const CompressCall& c, bool* applied);
 
 struct DecompressCall {
     const uint32_t* packed; uint64_t words_stride, words_valid; uint32_t n_workers; uint64_t d;

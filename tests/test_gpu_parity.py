@@ -238,6 +238,68 @@ def test_compress_tiled_copy_path_ragged_sizes(tq, orc, bits, mode, dtype):
     assert tq.tq_wait_expired_count() == 0
 
 
+@pytest.mark.parametrize("bits", [1, 2, 3, 4])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_compress_decision_table_path_ragged_sizes(tq, orc, bits, mode):
+    """bf16 rows of 2^18 elements and more take the kernel that reads the decision (interval and threshold)
+    from a per-block table indexed by the element's bit pattern: whole tiles, one element more, a partial
+    last run, several workers with a padded stride and different quantizers; salted with NaN of both signs,
+    Inf, +-alpha, zeros, subnormals and the levels themselves."""
+    L = 1 << bits
+    for d, n in ((262_144, 2), (262_145, 1), (262_176, 3), (270_337, 2), (300_003, 3)):
+        g = heavy_tailed(d, n, torch.bfloat16, seed=13 * bits + d)
+        ps = []
+        for i in range(n):
+            s = orc.stats(host_f32(orc, g[i, :d]), g_min=5e-4)
+            ls = tq.Stats(d=s.d, n_tail=max(s.n_tail, 100), n_nonfinite=0, sum_abs=s.sum_abs, sum_sq=s.sum_sq,
+                          sum_log_tail=max(s.sum_log_tail, 50.0), max_abs=max(s.max_abs, 0.05), g_min=5e-4)
+            ps.append(tq.tq_params(ls, L, mode, 3.0 + 0.25 * i))
+        salt_special_values(g, d, ps[0])
+        g[:, 5] = -float("nan")
+        g.view(torch.int16)[:, 6] = 0x7FFF                                               # NaN with the largest payload
+        g.view(torch.int16)[:, 7] = -1                                                   # the same with the sign set
+        g.view(torch.int16)[:, 8] = 1                                                    # smallest subnormal
+        g.view(torch.int16)[:, 9] = -32767                                               # its negative
+        seed, first = 0x9E3779B97F4A7C15, 2
+        words = tq.tq_packed_words(d, bits)
+        packed = torch.full((n, words + 8), 0x5A5A5A5A, dtype=torch.int32, device="cuda")
+        tq.tq_compress(g, ps, seed, first, d=d, packed=packed)
+        got = packed.cpu().numpy().view(np.uint32)
+        for i in range(n):
+            want = orc.compress(host_f32(orc, g[i, :d]), to_oracle_params(orc, ps[i]), seed, first + i)
+            assert np.array_equal(got[i, :words], want), (d, i)
+            assert np.all(got[i, words:] == 0x5A5A5A5A)
+
+
+def test_compress_decision_table_windows_and_fallback(tq, orc):
+    """The table covers a window of 16, 32 or 64 binades below alpha.  Codebooks whose scale puts the window
+    at the bottom of the exponent range, at its top, and whose central levels are too small for any window
+    (the element-wise kernel then runs) all give the oracle's codes; so does alpha = max|g| (no truncation)."""
+    d = 262_144 + 77
+    books = [
+        np.array([-1e-36, -3e-37, 2e-37, 1e-36], dtype=F32),                    # window reaches zero
+        np.array([-3e30, -1e30, -1e29, 1e28, 2e29, 5e29, 2e30, 3e30], dtype=F32),   # window high in the exponent range
+        np.array([-1.0, -1e-30, 1e-30, 1.0], dtype=F32),                         # no window: 100 binades between alpha and the centre
+        np.concatenate([[-2e-3], np.linspace(-1e-7, 1e-7, 14), [2e-3]]).astype(F32),   # crowded at zero, 64 binades
+        np.linspace(-0.75, 0.75, 16).astype(F32),
+    ]
+    for lv in books:
+        p = tq.tq_params_from_levels([float(x) for x in lv])
+        g = heavy_tailed(d, 2, torch.bfloat16, seed=len(lv), scale=float(lv[-1]) / 8)
+        salt_special_values(g, d, p)
+        got = tq.tq_compress(g, [p, p], seed=5, first_worker=1, d=d).cpu().numpy().view(np.uint32)
+        for i in range(2):
+            want = orc.compress(host_f32(orc, g[i, :d]), to_oracle_params(orc, p), 5, 1 + i)
+            assert np.array_equal(got[i], want), lv
+    g = heavy_tailed(d, 2, torch.bfloat16, seed=3)
+    st = tq.stats_to_host(tq.tq_stats(g, d))
+    for mode in (tq.UNIFORM, tq.NONUNIFORM):
+        ps = [tq.tq_params(s, 16, mode, 3.0, tq.ALPHA_MAXABS) for s in st]
+        got = tq.tq_compress(g, ps, seed=6, d=d).cpu().numpy().view(np.uint32)
+        for i in range(2):
+            assert np.array_equal(got[i], orc.compress(host_f32(orc, g[i, :d]), to_oracle_params(orc, ps[i]), 6, i))
+
+
 @pytest.mark.parametrize("bits,mode", [(2, 0), (3, 1), (4, 1), (4, 0)])
 def test_compress_million_elements_and_seed_sensitivity(tq, orc, bits, mode):
     d, n = 1_000_000 + 37, 2
