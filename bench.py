@@ -414,6 +414,56 @@ def measure_round(args, tq, w, g, stride, dev, local_rank, world, steps, warmup,
     if not headline:
         return result
 
+    # layer groups (Section 5): the round with the d elements cut into S equal groups, every step of it ONE launch
+    # over all (worker, group) pairs with the parameters designed on the device; and, for 16 groups, the same
+    # work as one set of calls per group
+    def equal_groups(S):
+        step = (d // S) // 16 * 16
+        return [(k * step, step if k < S - 1 else d - k * step) for k in range(S)]
+
+    def grouped_round(table, seg, sdev, wsd, pdev, pk):
+        tq.tq_stats_segments(g, seg, stats_dev=sdev, workspace=wsd)
+        tq.tq_params_device(sdev, N * len(table), w.num_levels, mode, w.gamma, params_dev=pdev)
+        tq.tq_compress_segments(g, seg, pdev, w.num_levels, mode, seed=1234, packed=pk)
+        tq.tq_decompress_aggregate_segments(pk, seg, pdev, w.num_levels, out=out)
+
+    def per_group_round(table, sdev, wsd, pdev, pk):
+        col = 0
+        for off, ln in table:
+            gv = g[:, off:off + ln]
+            wds = tq.tq_packed_words(ln, bits)
+            tq.tq_stats(gv, ln, stats_dev=sdev, workspace=wsd)
+            tq.tq_params_device(sdev, N, w.num_levels, mode, w.gamma, params_dev=pdev)
+            tq.tq_compress_device_params(gv, pdev, w.num_levels, mode, seed=1234, d=ln, packed=pk[:, col:col + wds])
+            tq.tq_decompress_aggregate_device_params(pk[:, col:col + wds], ln, pdev, w.num_levels, out=out[off:off + ln])
+            col += wds
+
+    def timed(fn, reps=20):
+        for _ in range(3):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    groups = {"round_ms": {}, "stats": "two passes (g_min = mean|g| of the group)", "params": "device"}
+    for S in (1, 4, 16, 64):
+        table = equal_groups(S)
+        seg = tq.segments_array(table)
+        sdev = torch.empty(N * S * 64, dtype=torch.uint8, device=dev)
+        wsd = torch.empty(tq.tq_stats_workspace_bytes(N * S), dtype=torch.uint8, device=dev)
+        pdev = torch.empty(N * S * 176, dtype=torch.uint8, device=dev)
+        pk = torch.empty((N, tq.tq_segments_packed_words(seg, bits)), dtype=torch.int32, device=dev)
+        groups["round_ms"][str(S)] = timed(lambda: grouped_round(table, seg, sdev, wsd, pdev, pk))
+        if S == 16:
+            groups["one_call_per_group_16_ms"] = timed(lambda: per_group_round(table, sdev, wsd, pdev, pk))
+        del sdev, wsd, pdev, pk
+    result["layer_groups"] = groups
+
     dom = "tq_compress"      # the single kernel with the largest share of the round (see profiles/launch_list_*)
     result["roofline"] = {"kernel": dom, "bound": "hbm", "achieved": kernels[dom]["gbs"], "peak": peak, "peak_source": peak_kind,
                           "unit": "GB/s", "frac": kernels[dom]["gbs"] / peak, "algorithmic_bytes": alg[dom][0],
@@ -589,6 +639,7 @@ def main():
             "roofline": head["roofline"], "kernels": head["kernels"], "cpu_baseline": head["cpu"], "e2e": head["e2e"],
             "gpu_launches": head["launches"], "clocks": head["clocks"],
             "update_checksum": head["checksum"],      # rank 0's aggregated update, for comparing variants
+            "layer_groups": head.get("layer_groups"),
             "workloads": workloads,
         }
         print(json.dumps(line), flush=True)

@@ -37,6 +37,7 @@ extern "C" {
 #define TQ_MAX_LEVELS 16
 #define TQ_MAX_WORKERS 64
 #define TQ_STATIC_MAX_WORKERS 16   /* most workers one tq_stats_static call can reduce */
+#define TQ_MAX_SEGMENTS 64         /* most layer groups per row in the tq_*_segments calls */
 
 typedef enum {
     TQ_OK = 0,
@@ -300,6 +301,47 @@ tq_status tq_compress_device_params(const void* grad_dev, tq_dtype dtype, uint64
 tq_status tq_decompress_aggregate_device_params(const uint32_t* packed_dev, size_t words_stride, uint32_t n_workers,
                                                 uint64_t d, const tq_params_t* params_dev, uint32_t num_levels,
                                                 const float* weights_host, float* out_dev, void* stream);
+
+/*
+ * Layer groups in one launch per step.  Section 5 (experimental setting) quantizes groups of layers --
+ * the convolutional and the fully-connected ones -- independently: each group has its own statistics,
+ * its own alpha and codebook, and its own packed stream.  A group is a segment [offset, offset + length)
+ * of every worker's row, the same for all workers.  These calls do for all (worker, segment) pairs at once
+ * what one tq_stats / tq_params_device / tq_compress_device_params / tq_decompress_aggregate_device_params
+ * call per group does on the sub-range, with the same results bit for bit:
+ *   - records are indexed [worker * n_segments + segment];
+ *   - element j of a segment is element j of that group's gradient: the random bits of Section 3.1's
+ *     rounding come from (seed, first_worker + worker, j) with j counted from the segment's start;
+ *   - segment s of a worker's packed row starts at word sum_{t < s} tq_packed_words(length_t, bits) of the row
+ *     (every segment is padded to a multiple of 4 words; tq_segments_packed_words gives the row total).
+ *   segments_host  [n_segments] host array, 1 <= n_segments <= TQ_MAX_SEGMENTS, read during the call; every
+ *                  length >= 1; offset * element size a multiple of 32 bytes (gradient: 8 fp32 or 16 bf16
+ *                  elements; output: 8 elements); segments must not overlap and, for the gradient, must end
+ *                  inside grad_stride.
+ *   n_workers * n_segments may reach TQ_MAX_WORKERS * TQ_MAX_SEGMENTS; tq_params_device accepts that many
+ *                  records.  tq_stats_segments needs tq_stats_workspace_bytes(n_workers * n_segments) of scratch.
+ * The parameter records are read from device memory (tq_params_device writes them there), so a round with
+ * layer groups needs no host round trip.  A pair whose statistics are outside the model's domain (for
+ * instance a one-element group) is marked TQ_FLAG_INVALID by tq_params_device; its packed segment is all
+ * zeros and it contributes zeros to the aggregate.
+ * Errors: INVALID_ARG (also overlapping or empty segments), ALIGNMENT, BUFFER_TOO_SMALL, CUDA.
+ */
+typedef struct {
+    uint64_t offset;   /* first element of the group in every worker's row */
+    uint64_t length;   /* elements */
+} tq_segment_t;
+size_t tq_segments_packed_words(const tq_segment_t* segments_host, uint32_t n_segments, uint32_t bits);
+tq_status tq_stats_segments(const void* grad_dev, tq_dtype dtype, uint64_t grad_stride, uint32_t n_workers,
+                            const tq_segment_t* segments_host, uint32_t n_segments, float g_min, float kappa,
+                            tq_stats_t* stats_dev, void* workspace_dev, size_t ws_bytes, void* stream);
+tq_status tq_compress_segments(const void* grad_dev, tq_dtype dtype, uint64_t grad_stride, uint32_t n_workers,
+                               const tq_segment_t* segments_host, uint32_t n_segments, const tq_params_t* params_dev,
+                               uint32_t num_levels, tq_mode mode, uint64_t seed, uint32_t first_worker,
+                               uint32_t* packed_dev, size_t words_stride, void* stream);
+tq_status tq_decompress_aggregate_segments(const uint32_t* packed_dev, size_t words_stride, uint32_t n_workers,
+                                           const tq_segment_t* segments_host, uint32_t n_segments,
+                                           const tq_params_t* params_dev, uint32_t num_levels,
+                                           const float* weights_host, float* out_dev, void* stream);
 
 const char* tq_strerror(tq_status status);
 int tq_last_cuda_error(void);   /* cudaError_t of the last failed runtime call on this thread, else 0 */

@@ -8,7 +8,7 @@ from __future__ import annotations
 import ctypes as C
 import math
 import os
-from typing import Optional, Sequence
+from typing import Optional, Sequence, Tuple
 
 import torch
 
@@ -27,7 +27,8 @@ FLAG_ALPHA_CAPPED, FLAG_ALPHA_AT_GMIN, FLAG_GAMMA_FROM_MLE, FLAG_INVALID = 1, 2,
 
 EXPORTS = ("tq_packed_words", "tq_stats_workspace_bytes", "tq_stats", "tq_stats_hinted", "tq_stats_static", "tq_params", "tq_params_batch", "tq_params_from_levels", "tq_params_device",
            "tq_compress_device_params", "tq_decompress_aggregate_device_params",
-           "tq_compress", "tq_decompress_aggregate", "tq_decompress_aggregate_rows", "tq_decompress_aggregate_apply", "tq_strerror", "tq_last_cuda_error", "tq_kernel_launches", "tq_wait_expired_count")
+           "tq_compress", "tq_decompress_aggregate", "tq_decompress_aggregate_rows", "tq_decompress_aggregate_apply",
+           "tq_segments_packed_words", "tq_stats_segments", "tq_compress_segments", "tq_decompress_aggregate_segments", "tq_strerror", "tq_last_cuda_error", "tq_kernel_launches", "tq_wait_expired_count")
 
 
 class Stats(C.Structure):
@@ -55,6 +56,11 @@ class TqError(RuntimeError):
 
 
 _lib: Optional[C.CDLL] = None
+
+
+class Segment(C.Structure):
+    """tq_segment_t: a layer group, [offset, offset + length) of every worker's row (elements)."""
+    _fields_ = [("offset", C.c_uint64), ("length", C.c_uint64)]
 
 
 def lib() -> C.CDLL:
@@ -92,6 +98,13 @@ def lib() -> C.CDLL:
         L.tq_decompress_aggregate_device_params.restype = C.c_int
         L.tq_decompress_aggregate_apply.argtypes = [vp, sz, u32, u64, C.POINTER(Params), C.POINTER(f32), vp, vp, f32, f32, f32, vp]
         L.tq_decompress_aggregate_apply.restype = C.c_int
+        L.tq_segments_packed_words.argtypes = [C.POINTER(Segment), u32, u32]; L.tq_segments_packed_words.restype = sz
+        L.tq_stats_segments.argtypes = [vp, C.c_int, u64, u32, C.POINTER(Segment), u32, f32, f32, vp, vp, sz, vp]
+        L.tq_stats_segments.restype = C.c_int
+        L.tq_compress_segments.argtypes = [vp, C.c_int, u64, u32, C.POINTER(Segment), u32, vp, u32, C.c_int, u64, u32, vp, sz, vp]
+        L.tq_compress_segments.restype = C.c_int
+        L.tq_decompress_aggregate_segments.argtypes = [vp, sz, u32, C.POINTER(Segment), u32, vp, u32, C.POINTER(f32), vp, vp]
+        L.tq_decompress_aggregate_segments.restype = C.c_int
         L.tq_strerror.argtypes = [C.c_int]; L.tq_strerror.restype = C.c_char_p
         L.tq_last_cuda_error.restype = C.c_int
         L.tq_kernel_launches.restype = u64
@@ -340,6 +353,60 @@ def tq_decompress_aggregate_device_params(packed: torch.Tensor, d: int, params_d
     _check(lib().tq_decompress_aggregate_device_params(packed.data_ptr(), words_stride, n, d, params_dev.data_ptr(),
                                                        num_levels, w, out.data_ptr(), _stream(stream)),
            "tq_decompress_aggregate_device_params")
+    return out
+
+
+def segments_array(segments: Sequence[Tuple[int, int]]):
+    """A tq_segment_t[n] from (offset, length) pairs."""
+    return (Segment * len(segments))(*[Segment(int(o), int(n)) for o, n in segments])
+
+
+def tq_segments_packed_words(segments, bits: int) -> int:
+    seg = segments if isinstance(segments, C.Array) else segments_array(segments)
+    return int(lib().tq_segments_packed_words(seg, len(seg), bits))
+
+
+def tq_stats_segments(grad: torch.Tensor, segments, g_min: float = 0.0, kappa: float = 1.0,
+                      stats_dev: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                      stream=None) -> torch.Tensor:
+    """One record per (worker, segment), index worker * n_segments + segment; returns the device records."""
+    n, _, stride = _grad_layout(grad, None)
+    seg = segments if isinstance(segments, C.Array) else segments_array(segments)
+    jobs = n * len(seg)
+    if stats_dev is None:
+        stats_dev = torch.empty(jobs * C.sizeof(Stats), dtype=torch.uint8, device=grad.device)
+    if workspace is None:
+        workspace = torch.empty(tq_stats_workspace_bytes(jobs), dtype=torch.uint8, device=grad.device)
+    _check(lib().tq_stats_segments(grad.data_ptr(), _dtype_code(grad), stride, n, seg, len(seg), g_min, kappa,
+                                   stats_dev.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream(stream)),
+           "tq_stats_segments")
+    return stats_dev
+
+
+def tq_compress_segments(grad: torch.Tensor, segments, params_dev: torch.Tensor, num_levels: int, mode: int, seed: int,
+                         first_worker: int = 0, packed: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    n, _, stride = _grad_layout(grad, None)
+    seg = segments if isinstance(segments, C.Array) else segments_array(segments)
+    bits = {2: 1, 4: 2, 8: 3, 16: 4}[num_levels]
+    if packed is None:
+        packed = torch.empty((n, tq_segments_packed_words(seg, bits)), dtype=torch.int32, device=grad.device)
+    words_stride = packed.stride(0) if packed.dim() == 2 and n > 1 else packed.shape[-1]
+    _check(lib().tq_compress_segments(grad.data_ptr(), _dtype_code(grad), stride, n, seg, len(seg), params_dev.data_ptr(),
+                                      num_levels, mode, seed & 0xFFFFFFFFFFFFFFFF, first_worker, packed.data_ptr(),
+                                      words_stride, _stream(stream)), "tq_compress_segments")
+    return packed
+
+
+def tq_decompress_aggregate_segments(packed: torch.Tensor, segments, params_dev: torch.Tensor, num_levels: int,
+                                     out: torch.Tensor, weights: Optional[Sequence[float]] = None, stream=None) -> torch.Tensor:
+    """Aggregates every segment into out[offset : offset + length]; elements of `out` outside the segments are left alone."""
+    n = packed.shape[0]
+    seg = segments if isinstance(segments, C.Array) else segments_array(segments)
+    w = None if weights is None else (C.c_float * n)(*[float(x) for x in weights])
+    words_stride = packed.stride(0) if n > 1 else packed.shape[1]
+    _check(lib().tq_decompress_aggregate_segments(packed.data_ptr(), words_stride, n, seg, len(seg), params_dev.data_ptr(),
+                                                  num_levels, w, out.data_ptr(), _stream(stream)),
+           "tq_decompress_aggregate_segments")
     return out
 
 

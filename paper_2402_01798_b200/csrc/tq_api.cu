@@ -170,7 +170,7 @@ tq_status tq_params_device(const tq_stats_t* stats_dev, uint32_t n_workers, uint
                            double gamma, tq_alpha_rule alpha_rule, double alpha_user, tq_params_t* params_dev,
                            void* stream) {
     uint32_t bits = 0;
-    if (!stats_dev || !params_dev || n_workers == 0 || n_workers > TQ_MAX_WORKERS) return TQ_ERR_INVALID_ARG;
+    if (!stats_dev || !params_dev || n_workers == 0 || n_workers > TQ_MAX_WORKERS * TQ_MAX_SEGMENTS) return TQ_ERR_INVALID_ARG;
     if (!tq::params_request_ok(num_levels, mode, alpha_rule, &bits)) return TQ_ERR_INVALID_ARG;
     if (alpha_rule == TQ_ALPHA_USER && !(alpha_user > 0.0)) return TQ_ERR_DOMAIN;
     if (!aligned(stats_dev, 8) || !aligned(params_dev, 8)) return TQ_ERR_ALIGNMENT;
@@ -236,6 +236,95 @@ tq_status tq_decompress_aggregate_apply(const uint32_t* packed_dev, size_t words
     tq::DecompressCall c{packed_dev, words_stride, need, n_workers, d, params_host, nullptr, weights_host, bits, nullptr,
                          static_cast<cudaStream_t>(stream)};
     c.theta = theta_dev; c.momentum_buf = momentum_dev; c.lr = lr; c.mu = momentum; c.wd = weight_decay;
+    const cudaError_t e = tq::launch_decompress(c);
+    if (e != cudaSuccess) return cuda_failed(e);
+    g_launches += 1;
+    return TQ_OK;
+}
+
+// ---- layer groups -------------------------------------------------------------------------------------
+
+static tq_status make_segments(const tq_segment_t* seg, uint32_t n_seg, uint32_t n_workers, uint64_t align_elems, uint32_t bits,
+                               uint64_t limit, tq::SegTable* out) {
+    if (!seg || n_seg == 0 || n_seg > TQ_MAX_SEGMENTS || n_workers == 0 || n_workers > TQ_MAX_WORKERS) return TQ_ERR_INVALID_ARG;
+    uint64_t words = 0;
+    out->n = n_seg; out->pad = 0;
+    for (uint32_t s = 0; s < n_seg; ++s) {
+        if (seg[s].length == 0 || seg[s].length > (1ull << 40) || seg[s].offset > (1ull << 40)) return TQ_ERR_INVALID_ARG;
+        if (seg[s].offset + seg[s].length > limit) return TQ_ERR_INVALID_ARG;
+        if (seg[s].offset % align_elems != 0) return TQ_ERR_ALIGNMENT;
+        for (uint32_t t = 0; t < s; ++t)
+            if (seg[s].offset < seg[t].offset + seg[t].length && seg[t].offset < seg[s].offset + seg[s].length) return TQ_ERR_INVALID_ARG;
+        out->off[s] = seg[s].offset; out->len[s] = seg[s].length; out->woff[s] = words;
+        words += bits ? tq_packed_words(seg[s].length, bits) : 0;
+    }
+    return TQ_OK;
+}
+
+size_t tq_segments_packed_words(const tq_segment_t* seg, uint32_t n_seg, uint32_t bits) {
+    if (!seg || bits < 1 || bits > 4) return 0;
+    size_t words = 0;
+    for (uint32_t s = 0; s < n_seg; ++s) words += tq_packed_words(seg[s].length, bits);
+    return words;
+}
+
+tq_status tq_stats_segments(const void* grad_dev, tq_dtype dtype, uint64_t grad_stride, uint32_t n_workers,
+                            const tq_segment_t* segments_host, uint32_t n_segments, float g_min, float kappa,
+                            tq_stats_t* stats_dev, void* workspace_dev, size_t ws_bytes, void* stream) {
+    if (tq_status s = check_grad(grad_dev, dtype, 1, grad_stride, n_workers)) return s;
+    static thread_local tq::SegTable segs;
+    if (tq_status s = make_segments(segments_host, n_segments, n_workers, 32 / elem_size(dtype), 0, grad_stride, &segs)) return s;
+    if (!stats_dev || !workspace_dev) return TQ_ERR_INVALID_ARG;
+    if (!(g_min > 0.0f) && !(kappa > 0.0f)) return TQ_ERR_INVALID_ARG;
+    if (!aligned(stats_dev, 8) || !aligned(workspace_dev, 256)) return TQ_ERR_ALIGNMENT;
+    if (ws_bytes < tq::stats_workspace_bytes(n_workers * n_segments)) return TQ_ERR_BUFFER_TOO_SMALL;
+    tq::StatsCall c{grad_dev, dtype == TQ_BF16, 0, grad_stride, n_workers, g_min, kappa, stats_dev, workspace_dev,
+                    static_cast<cudaStream_t>(stream)};
+    c.segs = &segs;
+    int launched = 0;
+    const cudaError_t e = tq::launch_stats(c, &launched);
+    g_launches += static_cast<uint64_t>(launched);
+    return e == cudaSuccess ? TQ_OK : cuda_failed(e);
+}
+
+tq_status tq_compress_segments(const void* grad_dev, tq_dtype dtype, uint64_t grad_stride, uint32_t n_workers,
+                               const tq_segment_t* segments_host, uint32_t n_segments, const tq_params_t* params_dev,
+                               uint32_t num_levels, tq_mode mode, uint64_t seed, uint32_t first_worker,
+                               uint32_t* packed_dev, size_t words_stride, void* stream) {
+    if (tq_status s = check_grad(grad_dev, dtype, 1, grad_stride, n_workers)) return s;
+    uint32_t bits = 0;
+    if (!params_dev || !tq::params_request_ok(num_levels, mode, TQ_ALPHA_CLOSED, &bits)) return TQ_ERR_INVALID_ARG;
+    static thread_local tq::SegTable segs;
+    if (tq_status s = make_segments(segments_host, n_segments, n_workers, 32 / elem_size(dtype), bits, grad_stride, &segs)) return s;
+    const size_t need = tq_segments_packed_words(segments_host, n_segments, bits);
+    if (!packed_dev) return TQ_ERR_INVALID_ARG;
+    if (!aligned(packed_dev, 16) || words_stride % 4 != 0 || !aligned(params_dev, 8)) return TQ_ERR_ALIGNMENT;
+    if (words_stride < need) return TQ_ERR_BUFFER_TOO_SMALL;
+    tq::CompressCall c{grad_dev, dtype == TQ_BF16, 0, grad_stride, n_workers, nullptr, params_dev, bits,
+                       mode != TQ_UNIFORM, seed, first_worker, packed_dev, words_stride, 0,
+                       static_cast<cudaStream_t>(stream)};
+    c.segs = &segs;
+    const cudaError_t e = tq::launch_compress(c);
+    if (e != cudaSuccess) return cuda_failed(e);
+    g_launches += mode != TQ_UNIFORM ? 2 : 1;
+    return TQ_OK;
+}
+
+tq_status tq_decompress_aggregate_segments(const uint32_t* packed_dev, size_t words_stride, uint32_t n_workers,
+                                           const tq_segment_t* segments_host, uint32_t n_segments,
+                                           const tq_params_t* params_dev, uint32_t num_levels,
+                                           const float* weights_host, float* out_dev, void* stream) {
+    uint32_t bits = 0;
+    if (!params_dev || !tq::params_request_ok(num_levels, TQ_UNIFORM, TQ_ALPHA_CLOSED, &bits)) return TQ_ERR_INVALID_ARG;
+    static thread_local tq::SegTable segs;
+    if (tq_status s = make_segments(segments_host, n_segments, n_workers, 8, bits, ~0ull, &segs)) return s;
+    const size_t need = tq_segments_packed_words(segments_host, n_segments, bits);
+    if (!packed_dev || !out_dev) return TQ_ERR_INVALID_ARG;
+    if (!aligned(packed_dev, 16) || words_stride % 4 != 0 || !aligned(out_dev, 32) || !aligned(params_dev, 8)) return TQ_ERR_ALIGNMENT;
+    if (words_stride < need) return TQ_ERR_BUFFER_TOO_SMALL;
+    tq::DecompressCall c{packed_dev, words_stride, 0, n_workers, 0, nullptr, params_dev, weights_host, bits, out_dev,
+                         static_cast<cudaStream_t>(stream)};
+    c.segs = &segs;
     const cudaError_t e = tq::launch_decompress(c);
     if (e != cudaSuccess) return cuda_failed(e);
     g_launches += 1;

@@ -379,18 +379,15 @@ __device__ __forceinline__ void build_tables(const WorkerQ& q, float2* s_grid, f
     if constexpr (!is_uniform(SEARCH)) __syncthreads();
 }
 
-// Per-block set-up of the shared tables for quantizer q, then the block's share of worker wi's runs.
+// Per-block set-up of the shared tables for quantizer q, then the block's share of the runs of one row
+// (`row`: its first gradient element, `prow`: its first packed word).
 // s_grid must hold kMaxGridCells + 1 entries when SEARCH == kGrid.
 template <int BITS, int SEARCH, bool BF16>
-__device__ __forceinline__ void compress_block(const WorkerQ& q, float2* s_grid, float2* s_cell, float* s_search,
-                                               const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
-                                               const RoundKeys& rk, uint32_t worker, uint32_t wi,
-                                               uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_out) {
+__device__ __forceinline__ void compress_row(const WorkerQ& q, float2* s_grid, float2* s_cell, float* s_search,
+                                             const char* __restrict__ row, uint64_t d, const RoundKeys& rk, uint32_t worker,
+                                             uint32_t* __restrict__ prow, uint64_t words_out) {
     build_tables<BITS, SEARCH>(q, s_grid, s_cell, s_search);
 
-    constexpr size_t esz = BF16 ? 2 : 4;
-    const char* row = static_cast<const char*>(grad) + static_cast<uint64_t>(wi) * grad_stride * esz;
-    uint32_t* prow = packed + static_cast<uint64_t>(wi) * words_stride;
     const uint64_t n_runs = (d + 31) >> 5;
     const RunCtx cx{q.alpha, q.inv_step, q.top, q.inv_2alpha, q.cell_scale, uniform_q<BITS>(q), reinterpret_cast<const char*>(s_grid),
                     reinterpret_cast<const char*>(s_cell), s_search};
@@ -402,6 +399,18 @@ __device__ __forceinline__ void compress_block(const WorkerQ& q, float2* s_grid,
         compress_run<BITS, SEARCH, BF16, false>(row, prow, run, d, words_out, worker, rk, cx);
     if (run == n_runs - 1)
         compress_run<BITS, SEARCH, BF16, true>(row, prow, run, d, words_out, worker, rk, cx);
+}
+
+// The same for worker wi's row of a [N][grad_stride] block and its row of the [N][words_stride] output.
+template <int BITS, int SEARCH, bool BF16>
+__device__ __forceinline__ void compress_block(const WorkerQ& q, float2* s_grid, float2* s_cell, float* s_search,
+                                               const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
+                                               const RoundKeys& rk, uint32_t worker, uint32_t wi,
+                                               uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_out) {
+    constexpr size_t esz = BF16 ? 2 : 4;
+    compress_row<BITS, SEARCH, BF16>(q, s_grid, s_cell, s_search,
+                                     static_cast<const char*>(grad) + static_cast<uint64_t>(wi) * grad_stride * esz, d, rk, worker,
+                                     packed + static_cast<uint64_t>(wi) * words_stride, words_out);
 }
 
 // Quantizers passed by value in the kernel's parameter space (host-side tq_params).
@@ -563,22 +572,42 @@ __device__ __forceinline__ void load_worker(const tq_params_t* __restrict__ para
     __syncthreads();
 }
 
+// Where a job's row and packed words are.  Without segments job wi is worker wi and its whole slice; with
+// segments it is the pair (worker, segment) = (wi / n, wi % n) and a piece of that worker's row.
+struct JobPlace {
+    const char* row; uint32_t* prow; uint64_t d, words_out; uint32_t worker;
+};
+template <int BITS, bool BF16>
+__device__ __forceinline__ JobPlace place_job(uint32_t wi, const void* grad, uint64_t d, uint64_t grad_stride, uint32_t first_worker,
+                                              uint32_t* packed, uint64_t words_stride, uint64_t words_out, const SegTable& segs) {
+    constexpr size_t esz = BF16 ? 2 : 4;
+    if (segs.n == 0)
+        return JobPlace{static_cast<const char*>(grad) + static_cast<uint64_t>(wi) * grad_stride * esz,
+                        packed + static_cast<uint64_t>(wi) * words_stride, d, words_out, first_worker + wi};
+    const uint32_t w = wi / segs.n, sg = wi - w * segs.n;
+    const uint64_t len = segs.len[sg];
+    return JobPlace{static_cast<const char*>(grad) + (static_cast<uint64_t>(w) * grad_stride + segs.off[sg]) * esz,
+                    packed + static_cast<uint64_t>(w) * words_stride + segs.woff[sg], len,
+                    (((len * BITS + 31) >> 5) + 3) & ~static_cast<uint64_t>(3), first_worker + w};
+}
+
 template <int BITS, bool NONUNIFORM, bool BF16>
 __global__ void __launch_bounds__(kThreads, TQ_COMPRESS_MIN_BLOCKS)
 compress_kernel_dev(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
                     const tq_params_t* __restrict__ params, const __grid_constant__ RoundKeys rk,
-                    uint32_t first_worker, uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_out) {
+                    uint32_t first_worker, uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_out,
+                    const __grid_constant__ SegTable segs) {
     __shared__ __align__(16) float2 s_grid[NONUNIFORM ? kMaxGridCells + 1 : 1];
     __shared__ __align__(16) float2 s_cell[TQ_MAX_LEVELS];
     __shared__ float s_search[2 * TQ_MAX_LEVELS];
     __shared__ WorkerQ s_q;
     const uint32_t wi = blockIdx.y;
+    const JobPlace job = place_job<BITS, BF16>(wi, grad, d, grad_stride, first_worker, packed, words_stride, words_out, segs);
     load_worker<BITS, NONUNIFORM>(params, wi, s_q);
     if (!(s_q.alpha > 0.0f)) {       // invalid parameters: the row is all code 0
-        uint32_t* prow = packed + static_cast<uint64_t>(wi) * words_stride;
-        for (uint64_t w = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x; w < words_out;
+        for (uint64_t w = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x; w < job.words_out;
              w += static_cast<uint64_t>(gridDim.x) * kThreads)
-            prow[w] = 0u;
+            job.prow[w] = 0u;
         return;
     }
     if constexpr (NONUNIFORM) {
@@ -586,29 +615,29 @@ compress_kernel_dev(const void* __restrict__ grad, uint64_t d, uint64_t grad_str
     }
     if constexpr (!NONUNIFORM) {
         if (s_q.inv_step_l == 0.0f) {    // alpha too large for the scaled inverse step
-            compress_block<BITS, kUniformWide, BF16>(s_q, s_grid, s_cell, s_search, grad, d, grad_stride, rk,
-                                                     first_worker + wi, wi, packed, words_stride, words_out);
+            compress_row<BITS, kUniformWide, BF16>(s_q, s_grid, s_cell, s_search, job.row, job.d, rk, job.worker, job.prow, job.words_out);
             return;
         }
     }
-    compress_block<BITS, NONUNIFORM ? kGrid : kUniform, BF16>(s_q, s_grid, s_cell, s_search, grad, d, grad_stride, rk,
-                                                              first_worker + wi, wi, packed, words_stride, words_out);
+    compress_row<BITS, NONUNIFORM ? kGrid : kUniform, BF16>(s_q, s_grid, s_cell, s_search, job.row, job.d, rk, job.worker, job.prow,
+                                                            job.words_out);
 }
 
 template <int BITS, bool BF16>
 __global__ void __launch_bounds__(kThreads, TQ_COMPRESS_MIN_BLOCKS)
 compress_kernel_dev_fallback(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
                              const tq_params_t* __restrict__ params, const __grid_constant__ RoundKeys rk,
-                             uint32_t first_worker, uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_out) {
+                             uint32_t first_worker, uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_out,
+                             const __grid_constant__ SegTable segs) {
     __shared__ __align__(16) float2 s_grid[1];
     __shared__ __align__(16) float2 s_cell[TQ_MAX_LEVELS];
     __shared__ float s_search[2 * TQ_MAX_LEVELS];
     __shared__ WorkerQ s_q;
     const uint32_t wi = blockIdx.y;
+    const JobPlace job = place_job<BITS, BF16>(wi, grad, d, grad_stride, first_worker, packed, words_stride, words_out, segs);
     load_worker<BITS, true>(params, wi, s_q);
     if (!(s_q.alpha > 0.0f) || s_q.cells != 0) return;
-    compress_block<BITS, kBinary, BF16>(s_q, s_grid, s_cell, s_search, grad, d, grad_stride, rk, first_worker + wi, wi,
-                                        packed, words_stride, words_out);
+    compress_row<BITS, kBinary, BF16>(s_q, s_grid, s_cell, s_search, job.row, job.d, rk, job.worker, job.prow, job.words_out);
 }
 
 // ---- host side ---------------------------------------------------------------------------------------
@@ -721,7 +750,7 @@ static cudaError_t dispatch(const CompressCall& c, const CompressArgs& a, dim3 g
 }
 
 cudaError_t launch_compress(const CompressCall& c) {
-    if (c.d == 0) return cudaSuccess;
+    if (c.d == 0 && !c.segs) return cudaSuccess;
     if (c.params_dev) return launch_compress_dev(c);
     {
         bool applied = false;
@@ -754,17 +783,20 @@ cudaError_t launch_compress(const CompressCall& c) {
     }
 }
 
+static const SegTable kNoSegments{};
+
 template <int BITS, bool NU, bool BF>
 static cudaError_t launch_dev(const CompressCall& c, dim3 grid) {
     const RoundKeys rk = round_keys(c.seed);
+    const SegTable& segs = c.segs ? *c.segs : kNoSegments;
     compress_kernel_dev<BITS, NU, BF><<<grid, kThreads, 0, c.stream>>>(
-        c.grad, c.d, c.grad_stride, c.params_dev, rk, c.first_worker, c.packed, c.words_stride, c.words_out);
+        c.grad, c.d, c.grad_stride, c.params_dev, rk, c.first_worker, c.packed, c.words_stride, c.words_out, segs);
     if constexpr (NU) {
         if (cudaError_t e = cudaGetLastError()) return e;
         // a small grid: this pass is empty unless a codebook is too crowded for the lookup grid
         const dim3 small(grid.x < 16 ? grid.x : 16, grid.y);
         compress_kernel_dev_fallback<BITS, BF><<<small, kThreads, 0, c.stream>>>(
-            c.grad, c.d, c.grad_stride, c.params_dev, rk, c.first_worker, c.packed, c.words_stride, c.words_out);
+            c.grad, c.d, c.grad_stride, c.params_dev, rk, c.first_worker, c.packed, c.words_stride, c.words_out, segs);
     }
     return cudaGetLastError();
 }
@@ -775,7 +807,15 @@ static cudaError_t dispatch_dev(const CompressCall& c, dim3 grid) {
 }
 
 cudaError_t launch_compress_dev(const CompressCall& c) {
-    const dim3 grid = compress_grid(c.d, c.n_workers, c.nonuniform);
+    // with segments: one grid row per (worker, segment) pair, sized by the longest segment
+    uint64_t d = c.d;
+    uint32_t jobs = c.n_workers;
+    if (c.segs) {
+        d = 0;
+        for (uint32_t sg = 0; sg < c.segs->n; ++sg) d = c.segs->len[sg] > d ? c.segs->len[sg] : d;
+        jobs = c.n_workers * c.segs->n;
+    }
+    const dim3 grid = compress_grid(d, jobs, c.nonuniform);
     switch (c.bits) {
         case 1: return dispatch_dev<1>(c, grid);
         case 2: return dispatch_dev<2>(c, grid);

@@ -35,6 +35,12 @@ struct DeviceTables {
     int use_weights;
     float weights[TQ_MAX_WORKERS];
 };
+// Layer groups: the tiles of all segments are numbered one after the other; segment sg owns tiles
+// tile_begin[sg] .. tile_begin[sg + 1] - 1 and worker i's codebook for it is params_dev[i * n + sg].
+struct SegTiles {
+    SegTable segs;
+    uint32_t tile_begin[TQ_MAX_SEGMENTS + 1];
+};
 
 __device__ __forceinline__ uint32_t ldg32_stream(const uint32_t* p) {
     uint32_t v;
@@ -195,12 +201,13 @@ __device__ __forceinline__ void finish_units(f32x2 (&acc)[Unit<BITS>::kUnits][Un
 }
 
 // Copies the N codebooks (already multiplied by w_i when weights are given) into shared memory.
-__device__ __forceinline__ void fill_tables(float* s_tab, uint32_t n, const DecompressArgs& args, const DeviceTables& dt) {
+__device__ __forceinline__ void fill_tables(float* s_tab, uint32_t n, const DecompressArgs& args, const DeviceTables& dt,
+                                            uint32_t pstride = 1, uint32_t poff = 0) {
     for (uint32_t t = threadIdx.x; t < n * TQ_MAX_LEVELS; t += kDecThreads) {
         const uint32_t i = t / TQ_MAX_LEVELS, k = t % TQ_MAX_LEVELS;
         float v;
         if (dt.params_dev) {     // same rounded product w_i * l as the host forms for the by-value table
-            const float l = dt.params_dev[i].levels[k];
+            const float l = dt.params_dev[i * pstride + poff].levels[k];
             v = dt.use_weights ? __fmul_rn(dt.weights[i], l) : l;
         } else {
             v = args.table[i][k];
@@ -322,9 +329,10 @@ __device__ __forceinline__ uint32_t stage_field(const uint32_t* seg, uint32_t ul
 
 template <int BITS, bool APPLY>
 __global__ void __launch_bounds__(kDecThreads, APPLY ? TQ_DECOMPRESS_BULK_BLOCKS - 2 : TQ_DECOMPRESS_BULK_BLOCKS)
-decompress_bulk_kernel(const __grid_constant__ RowTable rt, uint64_t words_valid, uint32_t n,
-                       uint64_t d, const __grid_constant__ DecompressArgs args, const __grid_constant__ DeviceTables dt,
-                       float scale, int divide, const __grid_constant__ ApplyArgs ap, float* __restrict__ out) {
+decompress_bulk_kernel(const __grid_constant__ RowTable rt, uint64_t words_row, uint32_t n,
+                       uint64_t d_row, const __grid_constant__ DecompressArgs args, const __grid_constant__ DeviceTables dt,
+                       float scale, int divide, const __grid_constant__ ApplyArgs ap_in, float* __restrict__ out_row,
+                       const __grid_constant__ SegTiles st) {
     constexpr int E = Unit<BITS>::kElems, U = Unit<BITS>::kUnits, S = TQ_DECOMPRESS_STAGES;
     constexpr uint32_t kSeg = Tile<BITS>::kSegBytes;
 
@@ -335,9 +343,25 @@ decompress_bulk_kernel(const __grid_constant__ RowTable rt, uint64_t words_valid
     const uint32_t stage0 = smem_addr(s_stage);
     const uint32_t bar0 = stage0 + S * kGroup * kSeg + 16;
 
-    const uint64_t tile = blockIdx.x;
-    const uint64_t tile_off = tile * kSeg;                                   // byte offset of the tile in every row
-    const uint64_t row_bytes = words_valid * 4;
+    // which stream this block decodes: the whole rows, or one segment of them
+    uint64_t tile = blockIdx.x, d = d_row, words_valid = words_row, row_shift = 0;    // row_shift: words from a row's start to the stream's
+    float* out = out_row;
+    ApplyArgs ap = ap_in;
+    uint32_t pstride = 1, poff = 0;
+    if (st.segs.n) {
+        uint32_t sg = 0;
+        while (sg + 1 < st.segs.n && st.tile_begin[sg + 1] <= blockIdx.x) ++sg;
+        tile = blockIdx.x - st.tile_begin[sg];
+        d = st.segs.len[sg];
+        words_valid = (((d * BITS + 31) >> 5) + 3) & ~static_cast<uint64_t>(3);
+        row_shift = st.segs.woff[sg];
+        if (out) out += st.segs.off[sg];
+        if (ap.theta) ap.theta += st.segs.off[sg];
+        if (ap.momentum_buf) ap.momentum_buf += st.segs.off[sg];
+        pstride = st.segs.n; poff = sg;
+    }
+    const uint64_t tile_off = tile * kSeg + row_shift * 4;                   // byte offset of the tile in every row
+    const uint64_t row_bytes = (words_valid + row_shift) * 4;
     const uint32_t seg_bytes = static_cast<uint32_t>(row_bytes - tile_off < kSeg ? row_bytes - tile_off : kSeg);
     const uint32_t n_steps = (n + kGroup - 1) / kGroup;
 
@@ -356,7 +380,7 @@ decompress_bulk_kernel(const __grid_constant__ RowTable rt, uint64_t words_valid
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         for (uint32_t q = 0; q < S && q < n_steps; ++q) issue(q);
     }
-    fill_tables(s_tab, n, args, dt);
+    fill_tables(s_tab, n, args, dt, pstride, poff);
     __syncthreads();          // barriers initialised and codebooks in place for every thread
     const char* tab_bytes = reinterpret_cast<const char*>(s_tab);
 
@@ -413,9 +437,11 @@ decompress_bulk_kernel(const __grid_constant__ RowTable rt, uint64_t words_valid
 // launch and set-up latency and keep the simpler direct kernel.
 constexpr uint64_t kBulkMinTiles = 8;
 
+static const SegTiles kNoSegTiles{};
+
 template <int BITS, bool APPLY>
 static cudaError_t launch_bulk(const DecompressCall& c, const RowTable& rt, const DecompressArgs& args, const DeviceTables& dt,
-                               float scale, int divide, const ApplyArgs& ap, uint64_t tiles) {
+                               float scale, int divide, const ApplyArgs& ap, uint64_t tiles, const SegTiles& st = kNoSegTiles) {
     const size_t smem = static_cast<size_t>(c.n_workers) * (kTabStride * 4) +
                         static_cast<size_t>(TQ_DECOMPRESS_STAGES) * kGroup * Tile<BITS>::kSegBytes + 16 + 8 * TQ_DECOMPRESS_STAGES;
     if (smem > 48 * 1024) {
@@ -424,13 +450,28 @@ static cudaError_t launch_bulk(const DecompressCall& c, const RowTable& rt, cons
         if (e != cudaSuccess) return e;
     }
     decompress_bulk_kernel<BITS, APPLY><<<static_cast<unsigned>(tiles), kDecThreads, smem, c.stream>>>(
-        rt, c.words_valid, c.n_workers, c.d, args, dt, scale, divide, ap, c.out);
+        rt, c.words_valid, c.n_workers, c.d, args, dt, scale, divide, ap, c.out, st);
     return cudaGetLastError();
 }
 
 template <int BITS>
 static cudaError_t launch(const DecompressCall& c, const RowTable& rt, const DecompressArgs& args, const DeviceTables& dt, float scale,
                           int divide) {
+    if (c.segs) {      // layer groups: the tiles of every segment in one grid, always through the bulk-copy kernel
+        static thread_local SegTiles st;
+        st.segs = *c.segs;
+        const uint64_t per_tile = static_cast<uint64_t>(kDecThreads) * Unit<BITS>::kUnits * Unit<BITS>::kElems;   // elements
+        uint64_t total = 0;
+        for (uint32_t sg = 0; sg < c.segs->n; ++sg) {
+            st.tile_begin[sg] = static_cast<uint32_t>(total);
+            total += (c.segs->len[sg] + per_tile - 1) / per_tile;
+            if (total > 0x7FFFFFFFull) return cudaErrorInvalidConfiguration;
+        }
+        st.tile_begin[c.segs->n] = static_cast<uint32_t>(total);
+        const ApplyArgs ap{c.theta, c.momentum_buf, c.lr, c.mu, c.wd};
+        return c.theta ? launch_bulk<BITS, true>(c, rt, args, dt, scale, divide, ap, total, st)
+                       : launch_bulk<BITS, false>(c, rt, args, dt, scale, divide, ap, total, st);
+    }
     const uint64_t n_units = (c.d + Unit<BITS>::kElems - 1) / Unit<BITS>::kElems;
     const uint64_t per_block = static_cast<uint64_t>(kDecThreads) * Unit<BITS>::kUnits;
     const uint64_t blocks = (n_units + per_block - 1) / per_block;

@@ -7,6 +7,17 @@
 
 namespace tq {
 
+// Layer groups (Section 5 quantizes groups of layers independently): every worker's row is cut into the same
+// n segments, and a (worker, segment) pair is handled like a worker of its own ("job" = worker * n + segment).
+// n = 0: no segments, a job is a worker and its row is the whole slice.
+struct SegTable {
+    uint32_t n;
+    uint32_t pad;
+    uint64_t off[TQ_MAX_SEGMENTS];    // first element of the segment in the row
+    uint64_t len[TQ_MAX_SEGMENTS];    // elements
+    uint64_t woff[TQ_MAX_SEGMENTS];   // first word of the segment's packed bits in the worker's packed row
+};
+
 struct CompressCall {
     const void* grad; bool bf16; uint64_t d, grad_stride; uint32_t n_workers;
     const tq_params_t* params;       // host array, or
@@ -15,6 +26,7 @@ struct CompressCall {
     uint64_t seed; uint32_t first_worker;
     uint32_t* packed; uint64_t words_stride, words_out;
     cudaStream_t stream;
+    const SegTable* segs = nullptr;  // device parameters only: params_dev[n_workers * segs->n]; d and words_out are then unused
 };
 cudaError_t launch_compress(const CompressCall& c);
 // bf16 rows through the per-bit-pattern decision table; *applied is false (and nothing is launched) when the
@@ -29,6 +41,7 @@ struct DecompressCall {
     float* out; cudaStream_t stream;
     float* theta = nullptr; float* momentum_buf = nullptr; float lr = 0.0f, mu = 0.0f, wd = 0.0f;   // fused model update
     const uint32_t* const* rows = nullptr;   // host array of n_workers row pointers; when set, packed / words_stride are unused
+    const SegTable* segs = nullptr;          // device parameters only: params_dev[n_workers * segs->n]; d and words_valid are then unused
 };
 cudaError_t launch_decompress(const DecompressCall& c);
 cudaError_t read_wait_expired(unsigned int* count);
@@ -37,6 +50,7 @@ cudaError_t read_compress_wait_expired(unsigned int* count);   // the same for t
 struct StatsCall {
     const void* grad; bool bf16; uint64_t d, grad_stride; uint32_t n_workers;
     float g_min, kappa; tq_stats_t* stats; void* workspace; cudaStream_t stream;
+    const SegTable* segs = nullptr;          // stats[n_workers * segs->n], workspace for that many jobs; d is then unused
 };
 // Enqueues the reduction; *launches receives the number of kernels launched.
 cudaError_t launch_stats(const StatsCall& c, int* launches);

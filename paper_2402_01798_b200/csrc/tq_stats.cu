@@ -52,11 +52,18 @@ __device__ __forceinline__ float fma_sat(float a, float b, float c) {
 
 template <bool BF16, int PASS>
 __global__ void __launch_bounds__(kThreads)
-stats_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride, float g_min_in, float kappa,
-             tq_stats_t* __restrict__ stats, Partial* __restrict__ partials, uint32_t* __restrict__ tickets) {
-    const uint32_t wi = blockIdx.y;
+stats_kernel(const void* __restrict__ grad, uint64_t d_row, uint64_t grad_stride, float g_min_in, float kappa,
+             tq_stats_t* __restrict__ stats, Partial* __restrict__ partials, uint32_t* __restrict__ tickets,
+             const __grid_constant__ SegTable segs) {
+    const uint32_t wi = blockIdx.y;          // the job: a worker, or a (worker, segment) pair
     const size_t esz = BF16 ? 2 : 4;
+    uint64_t d = d_row;
     const char* row = static_cast<const char*>(grad) + static_cast<uint64_t>(wi) * grad_stride * esz;
+    if (segs.n) {
+        const uint32_t worker = wi / segs.n, sg = wi - worker * segs.n;
+        row = static_cast<const char*>(grad) + (static_cast<uint64_t>(worker) * grad_stride + segs.off[sg]) * esz;
+        d = segs.len[sg];
+    }
 
     float g_min = g_min_in;
     if constexpr (PASS == kTail) g_min = stats[wi].g_min;     // finished by the moments pass
@@ -213,15 +220,25 @@ stats_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride, fl
     }
 }
 
+static const SegTable kNoSegments{};
+
 template <bool BF16, int PASS>
 static cudaError_t launch(const StatsCall& c, dim3 grid, Partial* partials, uint32_t* tickets) {
     stats_kernel<BF16, PASS><<<grid, kThreads, 0, c.stream>>>(c.grad, c.d, c.grad_stride, c.g_min, c.kappa,
-                                                              c.stats, partials, tickets);
+                                                              c.stats, partials, tickets, c.segs ? *c.segs : kNoSegments);
     return cudaGetLastError();
 }
 
-cudaError_t launch_stats(const StatsCall& c, int* launches) {
+cudaError_t launch_stats(const StatsCall& call, int* launches) {
     *launches = 0;
+    // with segments every (worker, segment) pair is a job of its own: same kernels, same scratch layout
+    StatsCall c = call;
+    const uint32_t n_jobs = c.segs ? c.n_workers * c.segs->n : c.n_workers;
+    if (c.segs) {
+        c.d = 0;
+        for (uint32_t sg = 0; sg < c.segs->n; ++sg) c.d = c.segs->len[sg] > c.d ? c.segs->len[sg] : c.d;   // sizes the grid
+    }
+    c.n_workers = n_jobs;
     Partial* partials = static_cast<Partial*>(c.workspace);
     uint32_t* tickets = reinterpret_cast<uint32_t*>(static_cast<char*>(c.workspace) + tickets_offset(c.n_workers));
     cudaError_t e = cudaMemsetAsync(tickets, 0, static_cast<size_t>(c.n_workers) * 2 * sizeof(uint32_t), c.stream);

@@ -235,6 +235,27 @@ def test_argument_validation_without_a_gpu(tq):
     assert L.tq_decompress_aggregate_rows(rows, 2, 64, mixed, None, ok_ptr, None) == tq.ERR_INVALID_ARG
     assert L.tq_decompress_aggregate_rows(rows, 2, 0, arr, None, ok_ptr, None) == tq.OK
     assert L.tq_wait_expired_count(None) == tq.ERR_INVALID_ARG
+    # layer groups: table checks come before any CUDA call
+    seg = tq.segments_array([(0, 100), (128, 60)])
+    ws2 = tq.tq_stats_workspace_bytes(2 * 2)
+    assert tq.tq_segments_packed_words(seg, 3) == tq.tq_packed_words(100, 3) + tq.tq_packed_words(60, 3)
+    assert L.tq_stats_segments(ok_ptr, tq.F32, 256, 2, None, 2, 0.0, 1.0, ok_ptr, ok_ptr, ws2, None) == tq.ERR_INVALID_ARG
+    assert L.tq_stats_segments(ok_ptr, tq.F32, 256, 2, seg, 0, 0.0, 1.0, ok_ptr, ok_ptr, ws2, None) == tq.ERR_INVALID_ARG
+    assert L.tq_stats_segments(ok_ptr, tq.F32, 256, 2, seg, 2, 0.0, 1.0, ok_ptr, ok_ptr, ws2 - 1, None) == tq.ERR_BUFFER_TOO_SMALL
+    assert L.tq_stats_segments(ok_ptr, tq.F32, 160, 2, seg, 2, 0.0, 1.0, ok_ptr, ok_ptr, ws2, None) == tq.ERR_INVALID_ARG      # second group ends past the row
+    assert L.tq_stats_segments(ok_ptr, tq.F32, 256, 2, tq.segments_array([(0, 100), (96, 8)]), 2, 0.0, 1.0, ok_ptr, ok_ptr, ws2, None) == tq.ERR_INVALID_ARG   # overlap
+    assert L.tq_stats_segments(ok_ptr, tq.F32, 256, 2, tq.segments_array([(0, 100), (100, 8)]), 2, 0.0, 1.0, ok_ptr, ok_ptr, ws2, None) == tq.ERR_ALIGNMENT
+    assert L.tq_stats_segments(ok_ptr, tq.BF16, 256, 2, tq.segments_array([(8, 64)]), 1, 0.0, 1.0, ok_ptr, ok_ptr, ws2, None) == tq.ERR_ALIGNMENT
+    assert L.tq_stats_segments(ok_ptr, tq.F32, 256, 2, tq.segments_array([(0, 0)]), 1, 0.0, 1.0, ok_ptr, ok_ptr, ws2, None) == tq.ERR_INVALID_ARG
+    need = tq.tq_segments_packed_words(seg, 3)
+    assert L.tq_compress_segments(ok_ptr, tq.F32, 256, 2, seg, 2, None, 8, tq.UNIFORM, 0, 0, ok_ptr, need, None) == tq.ERR_INVALID_ARG
+    assert L.tq_compress_segments(ok_ptr, tq.F32, 256, 2, seg, 2, ok_ptr, 7, tq.UNIFORM, 0, 0, ok_ptr, need, None) == tq.ERR_INVALID_ARG
+    assert L.tq_compress_segments(ok_ptr, tq.F32, 256, 2, seg, 2, ok_ptr, 8, tq.UNIFORM, 0, 0, ok_ptr, need - 4, None) == tq.ERR_BUFFER_TOO_SMALL
+    assert L.tq_compress_segments(ok_ptr, tq.F32, 256, 2, seg, 2, ok_ptr, 8, tq.UNIFORM, 0, 0, ok_ptr + 8, need, None) == tq.ERR_ALIGNMENT
+    assert L.tq_decompress_aggregate_segments(ok_ptr, need, 2, seg, 2, ok_ptr, 8, None, ok_ptr + 16, None) == tq.ERR_ALIGNMENT
+    assert L.tq_decompress_aggregate_segments(ok_ptr, need - 4, 2, seg, 2, ok_ptr, 8, None, ok_ptr, None) == tq.ERR_BUFFER_TOO_SMALL
+    assert L.tq_decompress_aggregate_segments(ok_ptr, need, 2, tq.segments_array([(4, 100)]), 1, ok_ptr, 8, None, ok_ptr, None) == tq.ERR_ALIGNMENT
+    assert L.tq_decompress_aggregate_segments(ok_ptr, need, 65, seg, 2, ok_ptr, 8, None, ok_ptr, None) == tq.ERR_INVALID_ARG
     # d = 0 needs no device at all
     assert L.tq_compress(ok_ptr, tq.F32, 0, 0, 1, arr, 0, 0, ok_ptr, 0, None) == tq.OK
     assert L.tq_decompress_aggregate(ok_ptr, 0, 1, 0, arr, None, ok_ptr, None) == tq.OK
