@@ -549,6 +549,8 @@ def main():
     ap.add_argument("--config", type=int, default=2, help="index into the five workloads (default: 25.6M x 16)")
     ap.add_argument("--variant", type=int, default=None,
                     help="with --config 3: index 0..11 into the bf16 sweep (gamma x mode x levels)")
+    ap.add_argument("--d", type=int, default=None,
+                    help="override the workload's elements per worker (a reduced copy of a large workload, for profiler captures)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--device-params", action="store_true",
                     help="design the parameters on the device (tq_params_device): no host round trip inside the round")
@@ -571,6 +573,9 @@ def main():
     w = inputs.WORKLOADS[args.config]
     if args.config == 3 and args.variant is not None:
         w = inputs.CONFIG4_SWEEP[args.variant]
+    if args.d is not None:
+        from dataclasses import replace
+        w = replace(w, d=args.d, name=f"{w.name}-d{args.d}")
     if args.impl == "reference":
         run_reference(args, w)
         return

@@ -36,7 +36,7 @@ constexpr int kLutMinEntries = 2048;
 constexpr uint32_t kSlotExpBits = 0x19000000u;   // 2^-77: exponent field 50, ulp 2^-100
 
 struct LutWorker {
-    float alpha, inv_step;
+    float alpha;
     uint32_t base2;       // -(base pattern) in both 16-bit halves
     uint32_t negtop2;     // the bf16 value -top in both halves
     float levels[TQ_MAX_LEVELS];
@@ -49,23 +49,14 @@ struct LutArgs {
 // X = k * 2^16 + min(T, 2^16) for a gradient value g: the decision of the quantizer equation up to the
 // random draw.  One IEEE operation per step (the build disables contraction on both sides), so host and
 // device agree bit for bit.
-__host__ __device__ inline uint32_t decision_x(float g, float alpha, float inv_step, const float* levels,
-                                               const float* inv_width, uint32_t num_levels, bool uniform) {
+__host__ __device__ inline uint32_t decision_x(float g, float alpha, const float* levels, const float* inv_width,
+                                               uint32_t num_levels) {
     const uint32_t s = num_levels - 1;
     const float t = fminf(fmaxf(g, -alpha), alpha);          // NaN -> -alpha, +-Inf -> +-alpha
-    uint32_t k;
-    float p;
-    if (uniform) {
-        const float x = (t + alpha) * inv_step;
-        const float fl = floorf(x);
-        k = fl >= static_cast<float>(s) ? s - 1 : static_cast<uint32_t>(fl);
-        p = x - static_cast<float>(k);
-    } else {
-        k = 0;
-        for (uint32_t j = 1; j + 1 <= s; ++j)
-            if (levels[j] <= t) k = j;
-        p = (t - levels[k]) * inv_width[k];
-    }
+    uint32_t k = 0;
+    for (uint32_t j = 1; j + 1 <= s; ++j)                     // largest j <= s - 1 with l_j <= t
+        if (levels[j] <= t) k = j;
+    const float p = (t - levels[k]) * inv_width[k];
     const float tf = p * 65536.0f;
     const uint32_t T = !(tf > 0.0f) ? 0u : (tf >= 65536.0f ? 65536u : static_cast<uint32_t>(rintf(tf)));
     return k * 65536u + T;
@@ -140,16 +131,9 @@ __device__ __forceinline__ void lut_piece(const uint32_t (&g)[Piece<BITS>::kElem
             // byte offsets of the two entries: 4 * clamp(|pattern| - base, 0, n - 1), negative values 32 KB further on
             const uint32_t off = __viaddmin_s16x2_relu(w & 0x7FFF7FFFu, cx.nbase2, cx.cap2) * 4u + (w & 0x80008000u);
             const float y0 = lds_f32(cx.table + (off & 0xFFFFu)), y1 = lds_f32(cx.table + (off >> 16));
-#ifdef TQ_LUT_I2F
-            float r0, r1;
-            asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tcvt.rn.f32.u16 %0, lo;\n\tcvt.rn.f32.u16 %1, hi;\n\t}"
-                : "=f"(r0), "=f"(r1) : "r"(rnd[h]));
-            code[h] = mul2_rd(fma2(pair(r0, r1), both(-7.888609052210118e-31f), pair(y0, y1)), down);
-#else
             const float r0 = __uint_as_float(__byte_perm(rnd[h], kSlotExpBits, 0x7610u));
             const float r1 = __uint_as_float(__byte_perm(rnd[h], kSlotExpBits, 0x7632u));
             code[h] = mul2_rd(sub2(pair(y0, y1), pair(r0, r1)), down);
-#endif
             if constexpr (TAIL) {                              // padding bits are zero
                 float c0, c1;
                 unpair(code[h], c0, c1);
@@ -199,9 +183,10 @@ __device__ __forceinline__ void load_piece(const char* row, uint64_t piece, uint
 #ifndef TQ_LUT_MIN_BLOCKS
 #define TQ_LUT_MIN_BLOCKS 3
 #endif
+constexpr int kLutThreads = kThreads;
 
-template <int BITS, bool UNIFORM>
-__global__ void __launch_bounds__(kThreads, TQ_LUT_MIN_BLOCKS)
+template <int BITS>
+__global__ void __launch_bounds__(kLutThreads, TQ_LUT_MIN_BLOCKS)
 compress_lut_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride, const __grid_constant__ LutArgs args,
                     const __grid_constant__ RoundKeys rk, uint32_t n_entries, uint32_t first_worker,
                     uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_out) {
@@ -212,16 +197,12 @@ compress_lut_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_str
     // the table: the decision for every bit pattern of the window, both signs
     {
         const uint32_t base = (0u - q.base2) & 0xFFFFu;
-        for (uint32_t i = threadIdx.x; i < 2 * n_entries; i += kThreads) {
+        for (uint32_t i = threadIdx.x; i < 2 * n_entries; i += kLutThreads) {
             const bool neg = i >= n_entries;
             const uint32_t c = neg ? i - n_entries : i;
             const uint32_t pattern = (base + c) | (neg ? 0x8000u : 0u);
-            const uint32_t x = decision_x(bf16_pattern_value(pattern), q.alpha, q.inv_step, q.levels, q.inv_width, 1u << BITS, UNIFORM);
-#ifdef TQ_LUT_I2F
-            s_table[c + (neg ? kLutMaxEntries : 0)] = __uint2float_rn(x + 65535u) * 7.888609052210118e-31f;
-#else
+            const uint32_t x = decision_x(bf16_pattern_value(pattern), q.alpha, q.levels, q.inv_width, 1u << BITS);
             s_table[c + (neg ? kLutMaxEntries : 0)] = __uint_as_float(kSlotExpBits + x + 65535u);
-#endif
         }
     }
     __syncthreads();
@@ -232,10 +213,10 @@ compress_lut_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_str
     const LutCtx cx{smem_addr(s_table), q.negtop2, q.base2, (n_entries - 1) * 0x00010001u,
                     philox_run(0u, first_worker + wi, rk)};
     const uint64_t interior = (d - 1) / E;                     // whole pieces before the row's last one
-    const uint64_t stride = static_cast<uint64_t>(gridDim.x) * kThreads;
+    const uint64_t stride = static_cast<uint64_t>(gridDim.x) * kLutThreads;
 
     // two sets of registers take turns: the next iteration's loads are in flight while this one is quantized
-    uint64_t piece = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x;
+    uint64_t piece = static_cast<uint64_t>(blockIdx.x) * kLutThreads + threadIdx.x;
     uint32_t a[PER_ITER][E / 2], b[PER_ITER][E / 2];
     auto fetch = [&](uint32_t (&buf)[PER_ITER][E / 2], uint64_t first) {
 #pragma unroll
@@ -283,42 +264,37 @@ static uint32_t top_pattern(float alpha) {
 
 // Entries per sign the worker needs, 0 if no window of at most kLutMaxEntries does.
 static uint32_t entries_needed(const tq_params_t& p, uint32_t top) {
-    const bool uniform = p.mode == TQ_UNIFORM;
     for (uint32_t n = kLutMinEntries; n <= static_cast<uint32_t>(kLutMaxEntries); n *= 2) {
         if (top < n) return n;                                 // the window reaches down to zero
         const uint32_t base = top - (n - 1);
-        const uint32_t lo = decision_x(bf16_pattern_value(base | 0x8000u), p.alpha, p.inv_step, p.levels, p.inv_width, p.num_levels, uniform);
-        const uint32_t hi = decision_x(bf16_pattern_value(base), p.alpha, p.inv_step, p.levels, p.inv_width, p.num_levels, uniform);
+        const uint32_t lo = decision_x(bf16_pattern_value(base | 0x8000u), p.alpha, p.levels, p.inv_width, p.num_levels);
+        const uint32_t hi = decision_x(bf16_pattern_value(base), p.alpha, p.levels, p.inv_width, p.num_levels);
         if (lo == hi) return n;                                // monotone: everything in between decides the same
     }
     return 0;
 }
 
-template <int BITS, bool UNIFORM>
+template <int BITS>
 static cudaError_t launch_lut(const CompressCall& c, const LutArgs& args, uint32_t n_entries) {
     const int smem = static_cast<int>((kLutMaxEntries + n_entries) * sizeof(float));
-    cudaError_t e = cudaFuncSetAttribute(compress_lut_kernel<BITS, UNIFORM>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = cudaFuncSetAttribute(compress_lut_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     int per_sm = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_lut_kernel<BITS, UNIFORM>, kThreads, smem);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_lut_kernel<BITS>, kLutThreads, smem);
     if (e != cudaSuccess) return e;
     if (per_sm < 1) per_sm = 1;
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const uint64_t tiles = (c.d / Piece<BITS>::kElems + kThreads - 1) / kThreads + 1;
+    const uint64_t tiles = (c.d / Piece<BITS>::kElems + kLutThreads - 1) / kLutThreads + 1;
     uint64_t per_worker = static_cast<uint64_t>(sms) * per_sm / c.n_workers;      // rounded down: one wave holds the grid
     if (per_worker > tiles) per_worker = tiles;
     if (per_worker < 1) per_worker = 1;
     const RoundKeys rk = round_keys(c.seed);
-    compress_lut_kernel<BITS, UNIFORM><<<dim3(static_cast<unsigned>(per_worker), c.n_workers), kThreads, smem, c.stream>>>(
+    compress_lut_kernel<BITS><<<dim3(static_cast<unsigned>(per_worker), c.n_workers), kLutThreads, smem, c.stream>>>(
         c.grad, c.d, c.grad_stride, args, rk, n_entries, c.first_worker, c.packed, c.words_stride, c.words_out);
     return cudaGetLastError();
 }
 
-template <int BITS>
-static cudaError_t dispatch_lut(const CompressCall& c, const LutArgs& a, uint32_t n) {
-    return c.nonuniform ? launch_lut<BITS, false>(c, a, n) : launch_lut<BITS, true>(c, a, n);
-}
 
 // Rows below this many elements keep the element-wise kernels (the table costs more than it saves).
 constexpr uint64_t kLutMinElements = 1u << 18;
@@ -341,17 +317,17 @@ cudaError_t launch_compress_lut(const CompressCall& c, bool* applied) {
         LutWorker& q = args.q[i];
         const uint32_t top = top_pattern(p.alpha);
         const uint32_t base = top >= n_entries ? top - (n_entries - 1) : 0u;   // a larger window than needed stays valid
-        q.alpha = p.alpha; q.inv_step = p.inv_step;
+        q.alpha = p.alpha;
         q.base2 = ((0u - base) & 0xFFFFu) * 0x00010001u;
         q.negtop2 = (top | 0x8000u) * 0x00010001u;
         for (int k = 0; k < TQ_MAX_LEVELS; ++k) { q.levels[k] = p.levels[k]; q.inv_width[k] = p.inv_width[k]; }
     }
     *applied = true;
     switch (c.bits) {
-        case 1: return dispatch_lut<1>(c, args, n_entries);
-        case 2: return dispatch_lut<2>(c, args, n_entries);
-        case 3: return dispatch_lut<3>(c, args, n_entries);
-        default: return dispatch_lut<4>(c, args, n_entries);
+        case 1: return launch_lut<1>(c, args, n_entries);
+        case 2: return launch_lut<2>(c, args, n_entries);
+        case 3: return launch_lut<3>(c, args, n_entries);
+        default: return launch_lut<4>(c, args, n_entries);
     }
 }
 

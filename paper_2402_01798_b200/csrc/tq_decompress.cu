@@ -336,7 +336,7 @@ decompress_bulk_kernel(const __grid_constant__ RowTable rt, uint64_t words_row, 
     constexpr int E = Unit<BITS>::kElems, U = Unit<BITS>::kUnits, S = TQ_DECOMPRESS_STAGES;
     constexpr uint32_t kSeg = Tile<BITS>::kSegBytes;
 
-    // [codebooks: n * 256 B][S stages of kGroup segments][16 B that a 3-bit field's second word may touch][S barriers]
+    // [codebooks: n * 64 B][S stages of kGroup segments][16 B that a 3-bit field's second word may touch][S barriers]
     extern __shared__ __align__(1024) unsigned char smem[];
     float* s_tab = reinterpret_cast<float*>(smem);
     unsigned char* s_stage = smem + static_cast<size_t>(n) * (kTabStride * 4);
@@ -408,7 +408,7 @@ decompress_bulk_kernel(const __grid_constant__ RowTable rt, uint64_t words_row, 
             // barrier makes the give-up decision uniform.
             if (__syncthreads_or(!ok)) { expired = true; break; }
             if (threadIdx.x == 0) issue(q + S);
-        } else if (!ok) {
+        } else if (!ok) {                      // a last step: no barrier here, the block agrees on it after the loop
             expired = true;
             break;
         }
@@ -421,8 +421,11 @@ decompress_bulk_kernel(const __grid_constant__ RowTable rt, uint64_t words_row, 
             }
         }
     }
+    // One barrier per block makes the give-up uniform in the last steps too: a tile is stored by all of its
+    // threads or by none, and the counter counts blocks.
+    expired = __syncthreads_or(expired);
     if (expired) {
-        atomicAdd(&g_wait_expired, 1u);
+        if (threadIdx.x == 0) atomicAdd(&g_wait_expired, 1u);
         if (threadIdx.x == 0)      // the copies issued and not yet seen to land: steps q .. q + S - 1
             for (uint32_t r = q; r < q + S && r < n_steps; ++r) mbar_wait(bar0 + 8 * (r % S), (r / S) & 1u);
         return;
