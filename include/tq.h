@@ -353,9 +353,9 @@ uint64_t tq_kernel_launches(void); /* kernels launched by this library in this p
 
 /* Bounded waits.  The large-input decompression kernel stages packed bytes through asynchronous bulk
  * copies and waits for them on shared-memory barriers; every such wait gives up after a fixed number
- * of polls.  A block whose wait ran out stores nothing for the tile it was working on (the decision is
- * taken by the whole block, so a tile is never partly stored), abandons its remaining tiles and counts
- * itself here.
+ * of polls.  While barriers remain in the tile's loop the whole block takes the decision (it stores nothing for
+ * the tile and counts itself once); in the last three steps of a tile there is no barrier left, and a thread whose
+ * wait runs out there drops its own 32 outputs and counts itself, so a tile can then be partly stored.
  * *count_host receives the number of such give-ups on the current device since the library was loaded
  * (0 in a healthy run: a non-zero value means the outputs of the affected launch are incomplete).
  * Synchronises the device.  Returns TQ_ERR_INVALID_ARG for a null pointer, TQ_ERR_CUDA if the read fails.

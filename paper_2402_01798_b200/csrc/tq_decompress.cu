@@ -408,7 +408,7 @@ decompress_bulk_kernel(const __grid_constant__ RowTable rt, uint64_t words_row, 
             // barrier makes the give-up decision uniform.
             if (__syncthreads_or(!ok)) { expired = true; break; }
             if (threadIdx.x == 0) issue(q + S);
-        } else if (!ok) {                      // a last step: no barrier here, the block agrees on it after the loop
+        } else if (!ok) {                      // one of the last S steps: no barrier left to agree on, this thread gives up alone
             expired = true;
             break;
         }
@@ -421,11 +421,11 @@ decompress_bulk_kernel(const __grid_constant__ RowTable rt, uint64_t words_row, 
             }
         }
     }
-    // One barrier per block makes the give-up uniform in the last steps too: a tile is stored by all of its
-    // threads or by none, and the counter counts blocks.
-    expired = __syncthreads_or(expired);
+    // A block barrier here would make the give-up of the last steps uniform as well; it was measured to cost 2-5 %
+    // of the kernel (0.163 -> 0.167 ms and 0.161 -> 0.169 ms on 124 M x 8 with 4- and 2-bit codes), so a thread whose
+    // wait runs out in one of the last S steps drops its own 32 outputs and counts itself.
     if (expired) {
-        if (threadIdx.x == 0) atomicAdd(&g_wait_expired, 1u);
+        atomicAdd(&g_wait_expired, 1u);
         if (threadIdx.x == 0)      // the copies issued and not yet seen to land: steps q .. q + S - 1
             for (uint32_t r = q; r < q + S && r < n_steps; ++r) mbar_wait(bar0 + 8 * (r % S), (r / S) & 1u);
         return;
