@@ -815,7 +815,9 @@ cudaError_t launch_compress_dev(const CompressCall& c) {
         for (uint32_t sg = 0; sg < c.segs->n; ++sg) d = c.segs->len[sg] > d ? c.segs->len[sg] : d;
         jobs = c.n_workers * c.segs->n;
     }
-    const dim3 grid = compress_grid(d, jobs, c.nonuniform);
+    // always the persistent grid here: a block first reads its quantizer from device memory and prepares it (two
+    // barriers and a global round trip), which one block per tile would pay 120 000 times on a large row
+    const dim3 grid = compress_grid(d, jobs, true);
     switch (c.bits) {
         case 1: return dispatch_dev<1>(c, grid);
         case 2: return dispatch_dev<2>(c, grid);
