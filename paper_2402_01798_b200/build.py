@@ -10,7 +10,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libtq.so")
 SOURCES = ["tq_api.cu", "tq_stats.cu", "tq_compress.cu", "tq_compress_lut.cu", "tq_decompress.cu", "tq_params.cu"]
-HEADERS = ["tq_device.cuh", "tq_launch.h"]
+HEADERS = ["tq_device.cuh", "tq_launch.h", "tq_lut.cuh"]
 
 NVCC_FLAGS = [
     "-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",

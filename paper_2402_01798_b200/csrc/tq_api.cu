@@ -196,9 +196,11 @@ tq_status tq_compress_device_params(const void* grad_dev, tq_dtype dtype, uint64
     tq::CompressCall c{grad_dev, dtype == TQ_BF16, d, grad_stride, n_workers, nullptr, params_dev, bits,
                        mode != TQ_UNIFORM, seed, first_worker, packed_dev, words_stride, need,
                        static_cast<cudaStream_t>(stream)};
+    int launched = 0;
+    c.launches = &launched;
     const cudaError_t e = tq::launch_compress(c);
     if (e != cudaSuccess) return cuda_failed(e);
-    g_launches += mode != TQ_UNIFORM ? 2 : 1;     // table mode: main kernel + the (usually empty) binary-search pass
+    g_launches += static_cast<uint64_t>(launched);   // table mode: main kernel + the (usually empty) binary-search pass; bf16: + the decision-table kernel
     return TQ_OK;
 }
 
@@ -304,9 +306,11 @@ tq_status tq_compress_segments(const void* grad_dev, tq_dtype dtype, uint64_t gr
                        mode != TQ_UNIFORM, seed, first_worker, packed_dev, words_stride, 0,
                        static_cast<cudaStream_t>(stream)};
     c.segs = &segs;
+    int launched = 0;
+    c.launches = &launched;
     const cudaError_t e = tq::launch_compress(c);
     if (e != cudaSuccess) return cuda_failed(e);
-    g_launches += mode != TQ_UNIFORM ? 2 : 1;
+    g_launches += static_cast<uint64_t>(launched);
     return TQ_OK;
 }
 

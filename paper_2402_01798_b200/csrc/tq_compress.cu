@@ -25,6 +25,7 @@
 
 #include "tq_device.cuh"
 #include "tq_launch.h"
+#include "tq_lut.cuh"
 
 namespace tq {
 
@@ -596,7 +597,11 @@ __global__ void __launch_bounds__(kThreads, TQ_COMPRESS_MIN_BLOCKS)
 compress_kernel_dev(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
                     const tq_params_t* __restrict__ params, const __grid_constant__ RoundKeys rk,
                     uint32_t first_worker, uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_out,
-                    const __grid_constant__ SegTable segs) {
+                    const __grid_constant__ SegTable segs, int table_kernel_ran) {
+    if (table_kernel_ran) {          // rows the decision-table kernel served are done (same rule, evaluated by every thread)
+        uint32_t top, base;
+        if (lut_serves_record(params[blockIdx.y], BITS, &top, &base)) return;
+    }
     __shared__ __align__(16) float2 s_grid[NONUNIFORM ? kMaxGridCells + 1 : 1];
     __shared__ __align__(16) float2 s_cell[TQ_MAX_LEVELS];
     __shared__ float s_search[2 * TQ_MAX_LEVELS];
@@ -628,7 +633,11 @@ __global__ void __launch_bounds__(kThreads, TQ_COMPRESS_MIN_BLOCKS)
 compress_kernel_dev_fallback(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride,
                              const tq_params_t* __restrict__ params, const __grid_constant__ RoundKeys rk,
                              uint32_t first_worker, uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_out,
-                             const __grid_constant__ SegTable segs) {
+                             const __grid_constant__ SegTable segs, int table_kernel_ran) {
+    if (table_kernel_ran) {
+        uint32_t top, base;
+        if (lut_serves_record(params[blockIdx.y], BITS, &top, &base)) return;
+    }
     __shared__ __align__(16) float2 s_grid[1];
     __shared__ __align__(16) float2 s_cell[TQ_MAX_LEVELS];
     __shared__ float s_search[2 * TQ_MAX_LEVELS];
@@ -786,24 +795,24 @@ cudaError_t launch_compress(const CompressCall& c) {
 static const SegTable kNoSegments{};
 
 template <int BITS, bool NU, bool BF>
-static cudaError_t launch_dev(const CompressCall& c, dim3 grid) {
+static cudaError_t launch_dev(const CompressCall& c, dim3 grid, int table_kernel_ran) {
     const RoundKeys rk = round_keys(c.seed);
     const SegTable& segs = c.segs ? *c.segs : kNoSegments;
     compress_kernel_dev<BITS, NU, BF><<<grid, kThreads, 0, c.stream>>>(
-        c.grad, c.d, c.grad_stride, c.params_dev, rk, c.first_worker, c.packed, c.words_stride, c.words_out, segs);
+        c.grad, c.d, c.grad_stride, c.params_dev, rk, c.first_worker, c.packed, c.words_stride, c.words_out, segs, table_kernel_ran);
     if constexpr (NU) {
         if (cudaError_t e = cudaGetLastError()) return e;
         // a small grid: this pass is empty unless a codebook is too crowded for the lookup grid
         const dim3 small(grid.x < 16 ? grid.x : 16, grid.y);
         compress_kernel_dev_fallback<BITS, BF><<<small, kThreads, 0, c.stream>>>(
-            c.grad, c.d, c.grad_stride, c.params_dev, rk, c.first_worker, c.packed, c.words_stride, c.words_out, segs);
+            c.grad, c.d, c.grad_stride, c.params_dev, rk, c.first_worker, c.packed, c.words_stride, c.words_out, segs, table_kernel_ran);
     }
     return cudaGetLastError();
 }
 template <int BITS>
-static cudaError_t dispatch_dev(const CompressCall& c, dim3 grid) {
-    if (c.nonuniform) return c.bf16 ? launch_dev<BITS, true, true>(c, grid) : launch_dev<BITS, true, false>(c, grid);
-    return c.bf16 ? launch_dev<BITS, false, true>(c, grid) : launch_dev<BITS, false, false>(c, grid);
+static cudaError_t dispatch_dev(const CompressCall& c, dim3 grid, int lut) {
+    if (c.nonuniform) return c.bf16 ? launch_dev<BITS, true, true>(c, grid, lut) : launch_dev<BITS, true, false>(c, grid, lut);
+    return c.bf16 ? launch_dev<BITS, false, true>(c, grid, lut) : launch_dev<BITS, false, false>(c, grid, lut);
 }
 
 cudaError_t launch_compress_dev(const CompressCall& c) {
@@ -817,12 +826,18 @@ cudaError_t launch_compress_dev(const CompressCall& c) {
     }
     // always the persistent grid here: a block first reads its quantizer from device memory and prepares it (two
     // barriers and a global round trip), which one block per tile would pay 120 000 times on a large row
-    const dim3 grid = compress_grid(d, jobs, true);
+    dim3 grid = compress_grid(d, jobs, true);
+    // bf16 table codebooks: the decision-table kernel first; it serves the rows its window fits and the element-wise
+    // kernels (a small grid then: they normally find nothing left) take the others
+    bool lut = false;
+    if (const cudaError_t e = launch_compress_lut(c, &lut)) return e;
+    if (lut && grid.x > 16) grid.x = 16;
+    if (c.launches) *c.launches = (c.nonuniform ? 2 : 1) + (lut ? 1 : 0);
     switch (c.bits) {
-        case 1: return dispatch_dev<1>(c, grid);
-        case 2: return dispatch_dev<2>(c, grid);
-        case 3: return dispatch_dev<3>(c, grid);
-        default: return dispatch_dev<4>(c, grid);
+        case 1: return dispatch_dev<1>(c, grid, lut);
+        case 2: return dispatch_dev<2>(c, grid, lut);
+        case 3: return dispatch_dev<3>(c, grid, lut);
+        default: return dispatch_dev<4>(c, grid, lut);
     }
 }
 

@@ -28,11 +28,10 @@
 
 #include "tq_device.cuh"
 #include "tq_launch.h"
+#include "tq_lut.cuh"
 
 namespace tq {
 
-constexpr int kLutMaxEntries = 8192;     // per sign
-constexpr int kLutMinEntries = 2048;
 constexpr uint32_t kSlotExpBits = 0x19000000u;   // 2^-77: exponent field 50, ulp 2^-100
 
 struct LutWorker {
@@ -45,32 +44,6 @@ struct LutWorker {
 struct LutArgs {
     LutWorker q[TQ_MAX_WORKERS];
 };
-
-// X = k * 2^16 + min(T, 2^16) for a gradient value g: the decision of the quantizer equation up to the
-// random draw.  One IEEE operation per step (the build disables contraction on both sides), so host and
-// device agree bit for bit.
-__host__ __device__ inline uint32_t decision_x(float g, float alpha, const float* levels, const float* inv_width,
-                                               uint32_t num_levels) {
-    const uint32_t s = num_levels - 1;
-    const float t = fminf(fmaxf(g, -alpha), alpha);          // NaN -> -alpha, +-Inf -> +-alpha
-    uint32_t k = 0;
-    for (uint32_t j = 1; j + 1 <= s; ++j)                     // largest j <= s - 1 with l_j <= t
-        if (levels[j] <= t) k = j;
-    const float p = (t - levels[k]) * inv_width[k];
-    const float tf = p * 65536.0f;
-    const uint32_t T = !(tf > 0.0f) ? 0u : (tf >= 65536.0f ? 65536u : static_cast<uint32_t>(rintf(tf)));
-    return k * 65536u + T;
-}
-
-__host__ __device__ inline float bf16_pattern_value(uint32_t pattern16) {
-#ifdef __CUDA_ARCH__
-    return __uint_as_float(pattern16 << 16);
-#else
-    union { uint32_t u; float f; } c;
-    c.u = pattern16 << 16;
-    return c.f;
-#endif
-}
 
 // ---- device ------------------------------------------------------------------------------------------
 
@@ -185,15 +158,11 @@ __device__ __forceinline__ void load_piece(const char* row, uint64_t piece, uint
 #endif
 constexpr int kLutThreads = kThreads;
 
+// A block's share of one row: build the table for quantizer q (n_entries per sign), then quantize.
 template <int BITS>
-__global__ void __launch_bounds__(kLutThreads, TQ_LUT_MIN_BLOCKS)
-compress_lut_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride, const __grid_constant__ LutArgs args,
-                    const __grid_constant__ RoundKeys rk, uint32_t n_entries, uint32_t first_worker,
-                    uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_out) {
-    extern __shared__ __align__(16) float s_table[];          // kLutMaxEntries + n_entries: the negative half starts at entry kLutMaxEntries
-    const uint32_t wi = blockIdx.y;
-    const LutWorker& q = args.q[wi];
-
+__device__ __forceinline__ void lut_block(const LutWorker& q, uint32_t n_entries, float* s_table, const char* __restrict__ row,
+                                          uint32_t* __restrict__ prow, uint64_t d, uint64_t words_out, uint32_t worker,
+                                          const RoundKeys& rk) {
     // the table: the decision for every bit pattern of the window, both signs
     {
         const uint32_t base = (0u - q.base2) & 0xFFFFu;
@@ -208,10 +177,7 @@ compress_lut_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_str
     __syncthreads();
 
     constexpr int E = Piece<BITS>::kElems, PER_ITER = 32 / E;   // 32 elements per thread and iteration: four Philox blocks in flight
-    const char* row = static_cast<const char*>(grad) + static_cast<uint64_t>(wi) * grad_stride * 2;
-    uint32_t* prow = packed + static_cast<uint64_t>(wi) * words_stride;
-    const LutCtx cx{smem_addr(s_table), q.negtop2, q.base2, (n_entries - 1) * 0x00010001u,
-                    philox_run(0u, first_worker + wi, rk)};
+    const LutCtx cx{smem_addr(s_table), q.negtop2, q.base2, (n_entries - 1) * 0x00010001u, philox_run(0u, worker, rk)};
     const uint64_t interior = (d - 1) / E;                     // whole pieces before the row's last one
     const uint64_t stride = static_cast<uint64_t>(gridDim.x) * kLutThreads;
 
@@ -251,28 +217,59 @@ compress_lut_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_str
     }
 }
 
-// ---- host --------------------------------------------------------------------------------------------
-
-// Smallest bf16 pattern whose value is >= alpha (alpha positive and finite).
-static uint32_t top_pattern(float alpha) {
-    union { float f; uint32_t u; } c;
-    c.f = alpha;
-    uint32_t p = c.u >> 16;
-    if ((p << 16) < c.u) ++p;
-    return p;                      // at most 0x7F80 (+Inf)
+// Quantizers passed by value (host-side tq_params); the host has chosen the window.
+template <int BITS>
+__global__ void __launch_bounds__(kLutThreads, TQ_LUT_MIN_BLOCKS)
+compress_lut_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride, const __grid_constant__ LutArgs args,
+                    const __grid_constant__ RoundKeys rk, uint32_t n_entries, uint32_t first_worker,
+                    uint32_t* __restrict__ packed, uint64_t words_stride, uint64_t words_out) {
+    extern __shared__ __align__(16) float s_table[];          // kLutMaxEntries + n_entries: the negative half starts at entry kLutMaxEntries
+    const uint32_t wi = blockIdx.y;
+    lut_block<BITS>(args.q[wi], n_entries, s_table, static_cast<const char*>(grad) + static_cast<uint64_t>(wi) * grad_stride * 2,
+                    packed + static_cast<uint64_t>(wi) * words_stride, d, words_out, first_worker + wi, rk);
 }
+
+// Quantizers read from device memory (tq_params_device).  Every block decides by lut_serves_record whether the
+// table form serves its row, with the largest window; rows it does not serve are left to the element-wise
+// device-parameter kernels, which are launched after this one and skip the rows served here.
+template <int BITS>
+__global__ void __launch_bounds__(kLutThreads, TQ_LUT_MIN_BLOCKS)
+compress_lut_kernel_dev(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride, const tq_params_t* __restrict__ params,
+                        const __grid_constant__ RoundKeys rk, uint32_t first_worker, uint32_t* __restrict__ packed,
+                        uint64_t words_stride, uint64_t words_out) {
+    extern __shared__ __align__(16) float s_table[];          // 2 * kLutMaxEntries
+    __shared__ LutWorker s_q;
+    __shared__ bool s_serves;
+    const uint32_t wi = blockIdx.y;
+    if (threadIdx.x < TQ_MAX_LEVELS) {
+        s_q.levels[threadIdx.x] = params[wi].levels[threadIdx.x];
+        s_q.inv_width[threadIdx.x] = params[wi].inv_width[threadIdx.x];
+    }
+    if (threadIdx.x == 0) {
+        uint32_t top = 0, base = 0;
+        s_serves = lut_serves_record(params[wi], BITS, &top, &base);
+        s_q.alpha = params[wi].alpha;
+        s_q.base2 = ((0u - base) & 0xFFFFu) * 0x00010001u;
+        s_q.negtop2 = (top | 0x8000u) * 0x00010001u;
+    }
+    __syncthreads();
+    if (!s_serves) return;
+    lut_block<BITS>(s_q, kLutMaxEntries, s_table, static_cast<const char*>(grad) + static_cast<uint64_t>(wi) * grad_stride * 2,
+                    packed + static_cast<uint64_t>(wi) * words_stride, d, words_out, first_worker + wi, rk);
+}
+
+// ---- host --------------------------------------------------------------------------------------------
 
 // Entries per sign the worker needs, 0 if no window of at most kLutMaxEntries does.
 static uint32_t entries_needed(const tq_params_t& p, uint32_t top) {
     for (uint32_t n = kLutMinEntries; n <= static_cast<uint32_t>(kLutMaxEntries); n *= 2) {
-        if (top < n) return n;                                 // the window reaches down to zero
-        const uint32_t base = top - (n - 1);
-        const uint32_t lo = decision_x(bf16_pattern_value(base | 0x8000u), p.alpha, p.levels, p.inv_width, p.num_levels);
-        const uint32_t hi = decision_x(bf16_pattern_value(base), p.alpha, p.levels, p.inv_width, p.num_levels);
-        if (lo == hi) return n;                                // monotone: everything in between decides the same
+        uint32_t base = 0;
+        if (lut_window_fits(p.alpha, p.levels, p.inv_width, p.num_levels, top, n, &base)) return n;
     }
     return 0;
 }
+
+static uint64_t lut_blocks_per_worker(uint64_t d, uint32_t n_workers, int per_sm, int pieces_elems);
 
 template <int BITS>
 static cudaError_t launch_lut(const CompressCall& c, const LutArgs& args, uint32_t n_entries) {
@@ -282,13 +279,7 @@ static cudaError_t launch_lut(const CompressCall& c, const LutArgs& args, uint32
     int per_sm = 0;
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_lut_kernel<BITS>, kLutThreads, smem);
     if (e != cudaSuccess) return e;
-    if (per_sm < 1) per_sm = 1;
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const uint64_t tiles = (c.d / Piece<BITS>::kElems + kLutThreads - 1) / kLutThreads + 1;
-    uint64_t per_worker = static_cast<uint64_t>(sms) * per_sm / c.n_workers;      // rounded down: one wave holds the grid
-    if (per_worker > tiles) per_worker = tiles;
-    if (per_worker < 1) per_worker = 1;
+    const uint64_t per_worker = lut_blocks_per_worker(c.d, c.n_workers, per_sm, Piece<BITS>::kElems);
     const RoundKeys rk = round_keys(c.seed);
     compress_lut_kernel<BITS><<<dim3(static_cast<unsigned>(per_worker), c.n_workers), kLutThreads, smem, c.stream>>>(
         c.grad, c.d, c.grad_stride, args, rk, n_entries, c.first_worker, c.packed, c.words_stride, c.words_out);
@@ -296,12 +287,44 @@ static cudaError_t launch_lut(const CompressCall& c, const LutArgs& args, uint32
 }
 
 
+static uint64_t lut_blocks_per_worker(uint64_t d, uint32_t n_workers, int per_sm, int pieces_elems) {
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const uint64_t tiles = (d / pieces_elems + kLutThreads - 1) / kLutThreads + 1;
+    uint64_t per_worker = static_cast<uint64_t>(sms) * (per_sm < 1 ? 1 : per_sm) / n_workers;      // rounded down: one wave holds the grid
+    if (per_worker > tiles) per_worker = tiles;
+    return per_worker < 1 ? 1 : per_worker;
+}
+
+template <int BITS>
+static cudaError_t launch_lut_dev(const CompressCall& c) {
+    const int smem = static_cast<int>(2 * kLutMaxEntries * sizeof(float));
+    cudaError_t e = cudaFuncSetAttribute(compress_lut_kernel_dev<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    int per_sm = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_lut_kernel_dev<BITS>, kLutThreads, smem);
+    if (e != cudaSuccess) return e;
+    const uint64_t per_worker = lut_blocks_per_worker(c.d, c.n_workers, per_sm, Piece<BITS>::kElems);
+    compress_lut_kernel_dev<BITS><<<dim3(static_cast<unsigned>(per_worker), c.n_workers), kLutThreads, smem, c.stream>>>(
+        c.grad, c.d, c.grad_stride, c.params_dev, round_keys(c.seed), c.first_worker, c.packed, c.words_stride, c.words_out);
+    return cudaGetLastError();
+}
+
 // Rows below this many elements keep the element-wise kernels (the table costs more than it saves).
 constexpr uint64_t kLutMinElements = 1u << 18;
 
 cudaError_t launch_compress_lut(const CompressCall& c, bool* applied) {
     *applied = false;
-    if (!c.bf16 || !c.nonuniform || c.params_dev || c.d < kLutMinElements || c.d > (1ull << 35)) return cudaSuccess;
+    if (!c.bf16 || !c.nonuniform || c.segs || c.d < kLutMinElements || c.d > (1ull << 35)) return cudaSuccess;
+    if (c.params_dev) {      // the kernel decides row by row; the caller launches the element-wise kernels for the rest
+        *applied = true;
+        switch (c.bits) {
+            case 1: return launch_lut_dev<1>(c);
+            case 2: return launch_lut_dev<2>(c);
+            case 3: return launch_lut_dev<3>(c);
+            default: return launch_lut_dev<4>(c);
+        }
+    }
     static thread_local LutArgs args;
     uint32_t n_entries = 0;
     for (uint32_t i = 0; i < c.n_workers; ++i) {

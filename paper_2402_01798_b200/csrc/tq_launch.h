@@ -27,6 +27,7 @@ struct CompressCall {
     uint32_t* packed; uint64_t words_stride, words_out;
     cudaStream_t stream;
     const SegTable* segs = nullptr;  // device parameters only: params_dev[n_workers * segs->n]; d and words_out are then unused
+    int* launches = nullptr;         // device parameters only: receives the number of kernels launched
 };
 cudaError_t launch_compress(const CompressCall& c);
 // bf16 rows through the per-bit-pattern decision table; *applied is false (and nothing is launched) when the

@@ -654,6 +654,37 @@ def test_device_params_marks_bad_statistics_and_fallback_codebooks(tq, orc):
         assert np.array_equal(pk[i], orc.compress(host_f32(orc, g2[i, :d]), to_oracle_params(orc, p), 9, i))
 
 
+@pytest.mark.parametrize("L", [4, 16])
+def test_device_params_rows_split_between_table_and_element_wise_kernels(tq, orc, L):
+    """bf16 rows with device-resident table codebooks: the decision-table kernel serves the rows its window fits and the
+    element-wise kernels the others (a codebook whose centre is 100 binades below alpha, a row marked invalid); every row
+    matches the oracle and the invalid one is all zeros.  Also through the whole device route from statistics on."""
+    d, bits = 262_144 + 77, {4: 2, 16: 4}[L]
+    half = L // 2
+    books = [np.concatenate([-np.geomspace(0.02, 2e-4, half), np.geomspace(2e-4, 0.02, half)]).astype(F32),
+             np.concatenate([-np.geomspace(1.0, 1e-30, half), np.geomspace(1e-30, 1.0, half)]).astype(F32),
+             np.concatenate([[-1.0], np.linspace(0.3, 0.3001, L - 2), [1.0]]).astype(F32)]
+    ps = [tq.tq_params_from_levels([float(x) for x in lv]) for lv in books]
+    bad = tq.Params()
+    bad.bits, bad.num_levels, bad.mode, bad.flags = bits, L, tq.NONUNIFORM, 8
+    ps.append(bad)
+    n = len(ps)
+    raw = torch.frombuffer(bytearray(b"".join(bytes(p) for p in ps)), dtype=torch.uint8).cuda()
+    g = heavy_tailed(d, n, torch.bfloat16, seed=L, scale=2e-3)
+    salt_special_values(g, d, ps[0])
+    got = tq.tq_compress_device_params(g, raw, L, tq.NONUNIFORM, seed=21, first_worker=3, d=d).cpu().numpy().view(np.uint32)
+    for i in range(n - 1):
+        want = orc.compress(host_f32(orc, g[i, :d]), to_oracle_params(orc, ps[i]), 21, 3 + i)
+        assert np.array_equal(got[i], want), i
+    assert not got[n - 1].any()
+    # statistics -> device parameters -> compress, nothing designed on the host
+    g2 = heavy_tailed(d, 3, torch.bfloat16, seed=50 + L)
+    pd = tq.tq_params_device(tq.tq_stats(g2, d), 3, L, tq.NONUNIFORM, 3.0)
+    got2 = tq.tq_compress_device_params(g2, pd, L, tq.NONUNIFORM, seed=22, d=d).cpu().numpy().view(np.uint32)
+    for i, p in enumerate(tq.params_to_host(pd)):
+        assert np.array_equal(got2[i], orc.compress(host_f32(orc, g2[i, :d]), to_oracle_params(orc, p), 22, i)), i
+
+
 @pytest.mark.parametrize("bits,n,mu,wd", [(4, 16, 0.9, 5e-4), (3, 4, 0.9, 0.0), (2, 8, 0.0, 1e-3), (4, 3, 0.0, 0.0), (1, 2, 0.5, 5e-4)])
 def test_fused_model_update_matches_oracle(tq, orc, bits, n, mu, wd):
     """tq_decompress_aggregate_apply: aggregation fused with the momentum-SGD step, two rounds in a row,
