@@ -300,6 +300,30 @@ def test_compress_decision_table_windows_and_fallback(tq, orc):
             assert np.array_equal(got[i], orc.compress(host_f32(orc, g[i, :d]), to_oracle_params(orc, ps[i]), 6, i))
 
 
+def test_compress_decision_table_many_workers_mixed_windows(tq, orc):
+    """64 workers in one launch whose codebooks need windows of different sizes (scales from 1e-20 to 1e30, centres
+    from close to alpha to 40 binades below it): the launch uses the largest window, every row still matches."""
+    d, n, L = 262_144 + 33, 64, 8
+    rng = np.random.default_rng(7)
+    ps, scales = [], []
+    for i in range(n):
+        a = float(10.0 ** rng.uniform(-20, 30))
+        inner = float(10.0 ** rng.uniform(-12, -0.3))
+        mags = np.geomspace(a * inner, a, L // 2).astype(F32)
+        ps.append(tq.tq_params_from_levels([float(x) for x in np.concatenate([-mags[::-1], mags])]))
+        scales.append(a)
+    from paper_2402_01798_b200 import inputs
+    stride = inputs.worker_stride(d, torch.bfloat16)
+    g = torch.zeros((n, stride), dtype=torch.bfloat16, device="cuda")
+    for i in range(n):
+        inputs.powerlaw_gradient(d, 3.0, scales[i] / 30, 900 + i, "cuda", torch.bfloat16, out=g[i, :d])
+    g[:, 11] = float("nan"); g[:, 12] = float("inf"); g[:, 13] = -float("inf"); g[:, 14] = 0.0
+    got = tq.tq_compress(g, ps, seed=99, first_worker=0, d=d).cpu().numpy().view(np.uint32)
+    for i in range(0, n, 3):
+        want = orc.compress(host_f32(orc, g[i, :d]), to_oracle_params(orc, ps[i]), 99, i)
+        assert np.array_equal(got[i], want), (i, scales[i])
+
+
 @pytest.mark.parametrize("bits,mode", [(2, 0), (3, 1), (4, 1), (4, 0)])
 def test_compress_million_elements_and_seed_sensitivity(tq, orc, bits, mode):
     d, n = 1_000_000 + 37, 2
