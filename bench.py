@@ -464,6 +464,30 @@ def measure_round(args, tq, w, g, stride, dev, local_rank, world, steps, warmup,
         del sdev, wsd, pdev, pk
     result["layer_groups"] = groups
 
+    # the whole round (one-pass statistics, device-made parameters: no host synchronisation inside) as ONE CUDA graph,
+    # against the same round launched kernel by kernel
+    def device_round():
+        run_stats(g)
+        tq.tq_params_device(stats_dev, N, w.num_levels, mode, w.gamma, params_dev=params_dev)
+        tq.tq_compress_device_params(g, params_dev, w.num_levels, mode, seed=1234, d=d, packed=packed)
+        tq.tq_decompress_aggregate_device_params(packed, d, params_dev, w.num_levels, out=out)
+
+    try:
+        launched = timed(device_round)
+        side = torch.cuda.Stream(device=dev)
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            device_round()                                   # every kernel loaded and configured before the capture
+        torch.cuda.current_stream().wait_stream(side)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            device_round()
+        result["cuda_graph"] = {"round_ms": timed(graph.replay), "launched_round_ms": launched,
+                                "what": "statistics (one pass) -> device parameters -> compress -> aggregate, captured once, replayed"}
+        del graph
+    except Exception as e:                                   # capture is an extra: report why it did not work
+        result["cuda_graph"] = {"error": repr(e)[:300]}
+
     dom = "tq_compress"      # the single kernel with the largest share of the round (see profiles/launch_list_*)
     result["roofline"] = {"kernel": dom, "bound": "hbm", "achieved": kernels[dom]["gbs"], "peak": peak, "peak_source": peak_kind,
                           "unit": "GB/s", "frac": kernels[dom]["gbs"] / peak, "algorithmic_bytes": alg[dom][0],
@@ -644,7 +668,7 @@ def main():
             "roofline": head["roofline"], "kernels": head["kernels"], "cpu_baseline": head["cpu"], "e2e": head["e2e"],
             "gpu_launches": head["launches"], "clocks": head["clocks"],
             "update_checksum": head["checksum"],      # rank 0's aggregated update, for comparing variants
-            "layer_groups": head.get("layer_groups"),
+            "layer_groups": head.get("layer_groups"), "cuda_graph": head.get("cuda_graph"),
             "workloads": workloads,
         }
         print(json.dumps(line), flush=True)

@@ -292,8 +292,9 @@ tq_status tq_decompress_aggregate_apply(const uint32_t* packed_dev, size_t words
  * tq_compress_device_params / tq_decompress_aggregate_device_params: as tq_compress /
  *   tq_decompress_aggregate with params_dev[n_workers] in device memory; bits and mode are not read
  *   from the records but given by the caller (num_levels, mode).
- * All three only enqueue work on `stream`.  Errors: INVALID_ARG, DOMAIN (alpha_user <= 0), ALIGNMENT,
- * BUFFER_TOO_SMALL, CUDA.
+ * All three only enqueue work on `stream`, so a round made of tq_stats_hinted (or tq_stats) and these three can be
+ * captured into a CUDA graph and replayed; call each once outside the capture first (the first launch of some kernels
+ * sets a function attribute).  Errors: INVALID_ARG, DOMAIN (alpha_user <= 0), ALIGNMENT, BUFFER_TOO_SMALL, CUDA.
  */
 tq_status tq_params_device(const tq_stats_t* stats_dev, uint32_t n_workers, uint32_t num_levels, tq_mode mode,
                            double gamma, tq_alpha_rule alpha_rule, double alpha_user, tq_params_t* params_dev,

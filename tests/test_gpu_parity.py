@@ -678,6 +678,48 @@ def test_device_params_marks_bad_statistics_and_fallback_codebooks(tq, orc):
         assert np.array_equal(pk[i], orc.compress(host_f32(orc, g2[i, :d]), to_oracle_params(orc, p), 9, i))
 
 
+@pytest.mark.parametrize("dtype,d", [(torch.float32, 300_007), (torch.bfloat16, 262_144 + 5)])
+def test_round_as_cuda_graph_replays_identically(tq, orc, dtype, d):
+    """The round without a host round trip (one-pass statistics, device-made parameters, compress, aggregate) captured once
+    as a CUDA graph: every replay on new data gives the packed rows and the update of the kernel-by-kernel round."""
+    n, L, mode = 4, 16, tq.NONUNIFORM
+    g = heavy_tailed(d, n, dtype, seed=5)
+    hint = tq.new_gmin_hint(n, "cuda")
+    stats_dev = torch.empty(n * 64, dtype=torch.uint8, device="cuda")
+    ws = torch.empty(tq.tq_stats_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+    params_dev = torch.empty(n * 176, dtype=torch.uint8, device="cuda")
+    packed = torch.empty((n, tq.tq_packed_words(d, 4)), dtype=torch.int32, device="cuda")
+    out = torch.empty(d, dtype=torch.float32, device="cuda")
+
+    def device_round():
+        tq.tq_stats_hinted(g, hint, d, stats_dev=stats_dev, workspace=ws)
+        tq.tq_params_device(stats_dev, n, L, mode, 3.0, params_dev=params_dev)
+        tq.tq_compress_device_params(g, params_dev, L, mode, seed=77, d=d, packed=packed)
+        tq.tq_decompress_aggregate_device_params(packed, d, params_dev, L, out=out)
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        device_round()                                   # warm-up outside the capture
+    torch.cuda.current_stream().wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        device_round()
+    for rnd in range(2):
+        g.copy_(heavy_tailed(d, n, dtype, seed=40 + rnd, scale=1e-3 * (1 + rnd)))      # new data, mean in another binade
+        graph.replay()
+        torch.cuda.synchronize()
+        got_packed, got_out = packed.clone(), out.clone()
+        ps = tq.params_to_host(params_dev)
+        device_round()
+        torch.cuda.synchronize()
+        assert torch.equal(got_packed, packed) and torch.equal(got_out, out)
+        for i in (0, n - 1):
+            want = orc.compress(host_f32(orc, g[i, :d]), to_oracle_params(orc, ps[i]), 77, i)
+            assert np.array_equal(got_packed[i].cpu().numpy().view(np.uint32), want)
+    assert tq.tq_wait_expired_count() == 0
+
+
 @pytest.mark.parametrize("L", [4, 16])
 def test_device_params_rows_split_between_table_and_element_wise_kernels(tq, orc, L):
     """bf16 rows with device-resident table codebooks: the decision-table kernel serves the rows its window fits and the
