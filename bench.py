@@ -56,7 +56,7 @@ class ClockSampler:
     """Samples SM clocks and throttle reasons through NVML (read-only) while the timed region runs."""
 
     def __init__(self, index: int, period_s: float = 0.001):
-        self.index, self.period, self.samples, self.reasons = index, period_s, [], set()
+        self.index, self.period, self.samples, self.reasons, self.mem_samples = index, period_s, [], set(), []
         self.max_mhz, self.stop_flag, self.thread, self.err = None, False, None, None
 
     def start(self):
@@ -84,6 +84,7 @@ class ClockSampler:
         while not self.stop_flag:
             try:
                 self.samples.append(float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                self.mem_samples.append(float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_MEM)))
                 mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
                 for nm, bit in names.items():
                     if mask & bit:
@@ -98,6 +99,7 @@ class ClockSampler:
         if self.thread:
             self.thread.join(timeout=2)
         out = {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz,
+               "mem_mhz": statistics.median(self.mem_samples) if self.mem_samples else None,
                "samples": len(self.samples), "reasons": sorted(self.reasons)}
         if self.err:
             out["error"] = self.err
@@ -371,7 +373,9 @@ def measure_round(args, tq, w, g, stride, dev, local_rank, world, steps, warmup,
     kernels = {"tq_params": dict(t_params, where="host (one sync)" if args.host_params else "device kernel")}
     # gbs / frac_of_hbm_peak from the mean over the timed steps; *_best from the fastest step
     kernels.update({k: dict(t, launches_per_step=n, algorithmic_bytes=b, gbs=b / (t["ms"] * 1e-3) / 1e9,
+                            input_gbs=in_bytes / (t["ms"] * 1e-3) / 1e9,      # bytes of gradient input of the round per second of this kernel
                             frac_of_hbm_peak=b / (t["ms"] * 1e-3) / 1e9 / peak,
+                            frac_of_nominal_8tbs=b / (t["ms"] * 1e-3) / 1e9 / 8000.0,
                             frac_of_hbm_peak_median=b / (t["ms_median"] * 1e-3) / 1e9 / peak,
                             frac_of_hbm_peak_best=b / (t["ms_min"] * 1e-3) / 1e9 / peak) for k, (b, t, n) in alg.items()})
 
