@@ -477,6 +477,8 @@ def measure_round(args, tq, w, g, stride, dev, local_rank, world, steps, warmup,
         tq.tq_decompress_aggregate_device_params(packed, d, params_dev, w.num_levels, out=out)
 
     try:
+        if world > 1:
+            raise RuntimeError("measured on one GPU only (a process group's watchdog thread may touch the device during a capture)")
         launched = timed(device_round)
         side = torch.cuda.Stream(device=dev)
         side.wait_stream(torch.cuda.current_stream())
@@ -484,7 +486,7 @@ def measure_round(args, tq, w, g, stride, dev, local_rank, world, steps, warmup,
             device_round()                                   # every kernel loaded and configured before the capture
         torch.cuda.current_stream().wait_stream(side)
         graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph):
+        with torch.cuda.graph(graph, capture_error_mode="thread_local"):
             device_round()
         result["cuda_graph"] = {"round_ms": timed(graph.replay), "launched_round_ms": launched,
                                 "what": "statistics (one pass) -> device parameters -> compress -> aggregate, captured once, replayed"}
