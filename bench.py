@@ -425,8 +425,11 @@ def measure_round(args, tq, w, g, stride, dev, local_rank, world, steps, warmup,
         step = (d // S) // 16 * 16
         return [(k * step, step if k < S - 1 else d - k * step) for k in range(S)]
 
-    def grouped_round(table, seg, sdev, wsd, pdev, pk):
-        tq.tq_stats_segments(g, seg, stats_dev=sdev, workspace=wsd)
+    def grouped_round(table, seg, sdev, wsd, pdev, pk, hnt=None):
+        if hnt is not None:
+            tq.tq_stats_hinted_segments(g, seg, hnt, stats_dev=sdev, workspace=wsd)
+        else:
+            tq.tq_stats_segments(g, seg, stats_dev=sdev, workspace=wsd)
         tq.tq_params_device(sdev, N * len(table), w.num_levels, mode, w.gamma, params_dev=pdev)
         tq.tq_compress_segments(g, seg, pdev, w.num_levels, mode, seed=1234, packed=pk)
         tq.tq_decompress_aggregate_segments(pk, seg, pdev, w.num_levels, out=out)
@@ -454,7 +457,8 @@ def measure_round(args, tq, w, g, stride, dev, local_rank, world, steps, warmup,
         torch.cuda.synchronize()
         return a.elapsed_time(b) / reps
 
-    groups = {"round_ms": {}, "stats": "two passes (g_min = mean|g| of the group)", "params": "device"}
+    groups = {"round_ms": {}, "round_ms_one_pass_stats": {}, "params": "device",
+              "stats": "round_ms: two passes (g_min = mean|g| of the group); round_ms_one_pass_stats: one hinted pass (power-of-two g_min)"}
     for S in (1, 4, 16, 64):
         table = equal_groups(S)
         seg = tq.segments_array(table)
@@ -463,6 +467,8 @@ def measure_round(args, tq, w, g, stride, dev, local_rank, world, steps, warmup,
         pdev = torch.empty(N * S * 176, dtype=torch.uint8, device=dev)
         pk = torch.empty((N, tq.tq_segments_packed_words(seg, bits)), dtype=torch.int32, device=dev)
         groups["round_ms"][str(S)] = timed(lambda: grouped_round(table, seg, sdev, wsd, pdev, pk))
+        hnt = tq.new_gmin_hint(N * S, dev)
+        groups["round_ms_one_pass_stats"][str(S)] = timed(lambda: grouped_round(table, seg, sdev, wsd, pdev, pk, hnt))
         if S == 16:
             groups["one_call_per_group_16_ms"] = timed(lambda: per_group_round(table, sdev, wsd, pdev, pk))
         del sdev, wsd, pdev, pk

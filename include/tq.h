@@ -339,6 +339,12 @@ size_t tq_segments_packed_words(const tq_segment_t* segments_host, uint32_t n_se
 tq_status tq_stats_segments(const void* grad_dev, tq_dtype dtype, uint64_t grad_stride, uint32_t n_workers,
                             const tq_segment_t* segments_host, uint32_t n_segments, float g_min, float kappa,
                             tq_stats_t* stats_dev, void* workspace_dev, size_t ws_bytes, void* stream);
+/* The one-pass statistics of tq_stats_hinted for every (worker, segment) pair: hint_dev holds n_workers * n_segments
+ * entries, indexed like the records; everything else as tq_stats_segments and tq_stats_hinted. */
+tq_status tq_stats_hinted_segments(const void* grad_dev, tq_dtype dtype, uint64_t grad_stride, uint32_t n_workers,
+                                   const tq_segment_t* segments_host, uint32_t n_segments, float kappa,
+                                   tq_gmin_hint_t* hint_dev, tq_stats_t* stats_dev, void* workspace_dev, size_t ws_bytes,
+                                   void* stream);
 tq_status tq_compress_segments(const void* grad_dev, tq_dtype dtype, uint64_t grad_stride, uint32_t n_workers,
                                const tq_segment_t* segments_host, uint32_t n_segments, const tq_params_t* params_dev,
                                uint32_t num_levels, tq_mode mode, uint64_t seed, uint32_t first_worker,

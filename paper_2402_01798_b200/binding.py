@@ -28,7 +28,7 @@ FLAG_ALPHA_CAPPED, FLAG_ALPHA_AT_GMIN, FLAG_GAMMA_FROM_MLE, FLAG_INVALID = 1, 2,
 EXPORTS = ("tq_packed_words", "tq_stats_workspace_bytes", "tq_stats", "tq_stats_hinted", "tq_stats_static", "tq_params", "tq_params_batch", "tq_params_from_levels", "tq_params_device",
            "tq_compress_device_params", "tq_decompress_aggregate_device_params",
            "tq_compress", "tq_decompress_aggregate", "tq_decompress_aggregate_rows", "tq_decompress_aggregate_apply",
-           "tq_segments_packed_words", "tq_stats_segments", "tq_compress_segments", "tq_decompress_aggregate_segments", "tq_strerror", "tq_last_cuda_error", "tq_kernel_launches", "tq_wait_expired_count")
+           "tq_segments_packed_words", "tq_stats_segments", "tq_stats_hinted_segments", "tq_compress_segments", "tq_decompress_aggregate_segments", "tq_strerror", "tq_last_cuda_error", "tq_kernel_launches", "tq_wait_expired_count")
 
 
 class Stats(C.Structure):
@@ -101,6 +101,8 @@ def lib() -> C.CDLL:
         L.tq_segments_packed_words.argtypes = [C.POINTER(Segment), u32, u32]; L.tq_segments_packed_words.restype = sz
         L.tq_stats_segments.argtypes = [vp, C.c_int, u64, u32, C.POINTER(Segment), u32, f32, f32, vp, vp, sz, vp]
         L.tq_stats_segments.restype = C.c_int
+        L.tq_stats_hinted_segments.argtypes = [vp, C.c_int, u64, u32, C.POINTER(Segment), u32, f32, vp, vp, vp, sz, vp]
+        L.tq_stats_hinted_segments.restype = C.c_int
         L.tq_compress_segments.argtypes = [vp, C.c_int, u64, u32, C.POINTER(Segment), u32, vp, u32, C.c_int, u64, u32, vp, sz, vp]
         L.tq_compress_segments.restype = C.c_int
         L.tq_decompress_aggregate_segments.argtypes = [vp, sz, u32, C.POINTER(Segment), u32, vp, u32, C.POINTER(f32), vp, vp]
@@ -380,6 +382,23 @@ def tq_stats_segments(grad: torch.Tensor, segments, g_min: float = 0.0, kappa: f
     _check(lib().tq_stats_segments(grad.data_ptr(), _dtype_code(grad), stride, n, seg, len(seg), g_min, kappa,
                                    stats_dev.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream(stream)),
            "tq_stats_segments")
+    return stats_dev
+
+
+def tq_stats_hinted_segments(grad: torch.Tensor, segments, hint: torch.Tensor, kappa: float = 1.0,
+                             stats_dev: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                             stream=None) -> torch.Tensor:
+    """tq_stats_hinted for every (worker, segment) pair; `hint` = new_gmin_hint(n_workers * n_segments), kept across rounds."""
+    n, _, stride = _grad_layout(grad, None)
+    seg = segments if isinstance(segments, C.Array) else segments_array(segments)
+    jobs = n * len(seg)
+    if stats_dev is None:
+        stats_dev = torch.empty(jobs * C.sizeof(Stats), dtype=torch.uint8, device=grad.device)
+    if workspace is None:
+        workspace = torch.empty(tq_stats_workspace_bytes(jobs), dtype=torch.uint8, device=grad.device)
+    _check(lib().tq_stats_hinted_segments(grad.data_ptr(), _dtype_code(grad), stride, n, seg, len(seg), kappa, hint.data_ptr(),
+                                          stats_dev.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream(stream)),
+           "tq_stats_hinted_segments")
     return stats_dev
 
 

@@ -289,6 +289,26 @@ tq_status tq_stats_segments(const void* grad_dev, tq_dtype dtype, uint64_t grad_
     return e == cudaSuccess ? TQ_OK : cuda_failed(e);
 }
 
+tq_status tq_stats_hinted_segments(const void* grad_dev, tq_dtype dtype, uint64_t grad_stride, uint32_t n_workers,
+                                   const tq_segment_t* segments_host, uint32_t n_segments, float kappa,
+                                   tq_gmin_hint_t* hint_dev, tq_stats_t* stats_dev, void* workspace_dev, size_t ws_bytes,
+                                   void* stream) {
+    if (tq_status s = check_grad(grad_dev, dtype, 1, grad_stride, n_workers)) return s;
+    static thread_local tq::SegTable segs;
+    if (tq_status s = make_segments(segments_host, n_segments, n_workers, 32 / elem_size(dtype), 0, grad_stride, &segs)) return s;
+    if (!stats_dev || !workspace_dev || !hint_dev) return TQ_ERR_INVALID_ARG;
+    if (!(kappa > 0.0f) || !(kappa <= 3.402823466e38f)) return TQ_ERR_INVALID_ARG;
+    if (!aligned(stats_dev, 8) || !aligned(hint_dev, 8) || !aligned(workspace_dev, 256)) return TQ_ERR_ALIGNMENT;
+    if (ws_bytes < tq::stats_workspace_bytes(n_workers * n_segments)) return TQ_ERR_BUFFER_TOO_SMALL;
+    tq::StatsCall c{grad_dev, dtype == TQ_BF16, 0, grad_stride, n_workers, 0.0f, kappa, stats_dev, workspace_dev,
+                    static_cast<cudaStream_t>(stream)};
+    c.segs = &segs;
+    int launched = 0;
+    const cudaError_t e = tq::launch_stats_hinted(c, hint_dev, &launched);
+    g_launches += static_cast<uint64_t>(launched);
+    return e == cudaSuccess ? TQ_OK : cuda_failed(e);
+}
+
 tq_status tq_compress_segments(const void* grad_dev, tq_dtype dtype, uint64_t grad_stride, uint32_t n_workers,
                                const tq_segment_t* segments_host, uint32_t n_segments, const tq_params_t* params_dev,
                                uint32_t num_levels, tq_mode mode, uint64_t seed, uint32_t first_worker,

@@ -298,16 +298,22 @@ __device__ __forceinline__ float pow2_floor(float x) {
 
 template <bool BF16, bool FALLBACK>
 __global__ void __launch_bounds__(kThreads, TQ_STATS_HINTED_BLOCKS)
-stats_hinted_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_stride, float kappa,
+stats_hinted_kernel(const void* __restrict__ grad, uint64_t d_row, uint64_t grad_stride, float kappa,
                     tq_gmin_hint_t* __restrict__ hint, tq_stats_t* __restrict__ stats,
-                    PartialH* __restrict__ partials, uint32_t* __restrict__ tickets) {
+                    PartialH* __restrict__ partials, uint32_t* __restrict__ tickets, const __grid_constant__ SegTable segs) {
     constexpr int K = FALLBACK ? 1 : 2;
-    const uint32_t wi = blockIdx.y;
+    const uint32_t wi = blockIdx.y;               // the job: a worker, or a (worker, segment) pair
     if constexpr (FALLBACK) {
         if (hint[wi].hit) return;                 // the one-pass result stands
     }
     const size_t esz = BF16 ? 2 : 4;
+    uint64_t d = d_row;
     const char* row = static_cast<const char*>(grad) + static_cast<uint64_t>(wi) * grad_stride * esz;
+    if (segs.n) {
+        const uint32_t worker = wi / segs.n, sg = wi - worker * segs.n;
+        row = static_cast<const char*>(grad) + (static_cast<uint64_t>(worker) * grad_stride + segs.off[sg]) * esz;
+        d = segs.len[sg];
+    }
 
     // candidate thresholds
     float t[2] = {CUDART_INF_F, CUDART_INF_F};
@@ -512,8 +518,15 @@ stats_hinted_kernel(const void* __restrict__ grad, uint64_t d, uint64_t grad_str
     }
 }
 
-cudaError_t launch_stats_hinted(const StatsCall& c, tq_gmin_hint_t* hint, int* launches) {
+cudaError_t launch_stats_hinted(const StatsCall& call, tq_gmin_hint_t* hint, int* launches) {
     *launches = 0;
+    StatsCall c = call;                          // with segments every (worker, segment) pair is a job of its own
+    if (c.segs) {
+        c.d = 0;
+        for (uint32_t sg = 0; sg < c.segs->n; ++sg) c.d = c.segs->len[sg] > c.d ? c.segs->len[sg] : c.d;   // sizes the grid
+        c.n_workers *= c.segs->n;
+    }
+    const SegTable& segs = c.segs ? *c.segs : kNoSegments;
     PartialH* partials = static_cast<PartialH*>(c.workspace);
     uint32_t* tickets = reinterpret_cast<uint32_t*>(static_cast<char*>(c.workspace) + tickets_offset(c.n_workers));
     cudaError_t e = cudaMemsetAsync(tickets, 0, static_cast<size_t>(c.n_workers) * 2 * sizeof(uint32_t), c.stream);
@@ -528,13 +541,13 @@ cudaError_t launch_stats_hinted(const StatsCall& c, tq_gmin_hint_t* hint, int* l
     if (per_worker > kMaxBlocksPerWorker) per_worker = kMaxBlocksPerWorker;
     if (per_worker < 1) per_worker = 1;
     const dim3 grid(static_cast<unsigned>(per_worker), c.n_workers);     // the same grid for both kernels: same summation order
-    if (c.bf16) stats_hinted_kernel<true, false><<<grid, kThreads, 0, c.stream>>>(c.grad, c.d, c.grad_stride, c.kappa, hint, c.stats, partials, tickets);
-    else stats_hinted_kernel<false, false><<<grid, kThreads, 0, c.stream>>>(c.grad, c.d, c.grad_stride, c.kappa, hint, c.stats, partials, tickets);
+    if (c.bf16) stats_hinted_kernel<true, false><<<grid, kThreads, 0, c.stream>>>(c.grad, c.d, c.grad_stride, c.kappa, hint, c.stats, partials, tickets, segs);
+    else stats_hinted_kernel<false, false><<<grid, kThreads, 0, c.stream>>>(c.grad, c.d, c.grad_stride, c.kappa, hint, c.stats, partials, tickets, segs);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     *launches = 1;
-    if (c.bf16) stats_hinted_kernel<true, true><<<grid, kThreads, 0, c.stream>>>(c.grad, c.d, c.grad_stride, c.kappa, hint, c.stats, partials, tickets);
-    else stats_hinted_kernel<false, true><<<grid, kThreads, 0, c.stream>>>(c.grad, c.d, c.grad_stride, c.kappa, hint, c.stats, partials, tickets);
+    if (c.bf16) stats_hinted_kernel<true, true><<<grid, kThreads, 0, c.stream>>>(c.grad, c.d, c.grad_stride, c.kappa, hint, c.stats, partials, tickets, segs);
+    else stats_hinted_kernel<false, true><<<grid, kThreads, 0, c.stream>>>(c.grad, c.d, c.grad_stride, c.kappa, hint, c.stats, partials, tickets, segs);
     e = cudaGetLastError();
     if (e == cudaSuccess) *launches = 2;
     return e;

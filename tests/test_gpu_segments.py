@@ -154,6 +154,34 @@ def test_segments_with_weights_and_many_pairs(tq, orc):
         assert np.array_equal(res[off:off + x], agg)
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("table", [TWO_GROUPS, SIXTEEN], ids=["two", "sixteen"])
+def test_one_pass_statistics_per_segment(tq, orc, dtype, table):
+    """tq_stats_hinted_segments: per (worker, segment) the record of the oracle under the power-of-two threshold rule,
+    whether the hint is missing, fresh or stale (the record does not depend on it, bit for bit)."""
+    n, width = 3, 200_000
+    g = make_rows(n, width, dtype, seed=17)
+    S = len(table)
+    hint = tq.new_gmin_hint(n * S, "cuda")
+    first = tq.stats_to_host(tq.tq_stats_hinted_segments(g, table, hint))           # no hint: every pair takes the tail pass
+    again = tq.stats_to_host(tq.tq_stats_hinted_segments(g, table, hint))           # hint from the same data: one pass
+    hits = [hit for _, hit in tq.gmin_hint_to_host(hint)]
+    for i in range(n):
+        for s, (off, ln) in enumerate(table):
+            a, b = first[i * S + s], again[i * S + s]
+            assert bytes(a) == bytes(b), (i, s)
+            o = orc.stats_pow2(host_f32(orc, g[i, off:off + ln]))
+            assert a.d == ln and a.g_min == o.g_min and a.n_tail == o.n_tail and a.max_abs == o.max_abs
+            assert math.isclose(a.sum_abs, o.sum_abs, rel_tol=TOL_SUM)
+            assert math.isclose(a.sum_log_tail, o.sum_log_tail, rel_tol=TOL_LOG, abs_tol=1e-9)
+            if a.g_min > 0:
+                assert hits[i * S + s] == 1
+    g2 = (g.float() * 37.0).to(dtype)                                                # the mean moves five binades: stale hints
+    stale = tq.stats_to_host(tq.tq_stats_hinted_segments(g2, table, hint))
+    fresh = tq.stats_to_host(tq.tq_stats_hinted_segments(g2, table, tq.new_gmin_hint(n * S, "cuda")))
+    assert all(bytes(x) == bytes(y) for x, y in zip(stale, fresh))
+
+
 def test_segment_argument_checks(tq):
     g = torch.zeros((2, 4096), dtype=torch.float32, device="cuda")
     for bad, status in (([(0, 0)], tq.ERR_INVALID_ARG), ([(4, 100)], tq.ERR_ALIGNMENT), ([(0, 100), (96, 50)], tq.ERR_INVALID_ARG),
