@@ -247,6 +247,10 @@ def test_argument_validation_without_a_gpu(tq):
     assert L.tq_stats_segments(ok_ptr, tq.F32, 256, 2, tq.segments_array([(0, 100), (100, 8)]), 2, 0.0, 1.0, ok_ptr, ok_ptr, ws2, None) == tq.ERR_ALIGNMENT
     assert L.tq_stats_segments(ok_ptr, tq.BF16, 256, 2, tq.segments_array([(8, 64)]), 1, 0.0, 1.0, ok_ptr, ok_ptr, ws2, None) == tq.ERR_ALIGNMENT
     assert L.tq_stats_segments(ok_ptr, tq.F32, 256, 2, tq.segments_array([(0, 0)]), 1, 0.0, 1.0, ok_ptr, ok_ptr, ws2, None) == tq.ERR_INVALID_ARG
+    assert L.tq_stats_hinted_segments(ok_ptr, tq.F32, 256, 2, seg, 2, 1.0, None, ok_ptr, ok_ptr, ws2, None) == tq.ERR_INVALID_ARG
+    assert L.tq_stats_hinted_segments(ok_ptr, tq.F32, 256, 2, seg, 2, 0.0, ok_ptr, ok_ptr, ok_ptr, ws2, None) == tq.ERR_INVALID_ARG
+    assert L.tq_stats_hinted_segments(ok_ptr, tq.F32, 256, 2, seg, 2, 1.0, ok_ptr + 4, ok_ptr, ok_ptr, ws2, None) == tq.ERR_ALIGNMENT
+    assert L.tq_stats_hinted_segments(ok_ptr, tq.F32, 256, 2, seg, 2, 1.0, ok_ptr, ok_ptr, ok_ptr, ws2 - 1, None) == tq.ERR_BUFFER_TOO_SMALL
     need = tq.tq_segments_packed_words(seg, 3)
     assert L.tq_compress_segments(ok_ptr, tq.F32, 256, 2, seg, 2, None, 8, tq.UNIFORM, 0, 0, ok_ptr, need, None) == tq.ERR_INVALID_ARG
     assert L.tq_compress_segments(ok_ptr, tq.F32, 256, 2, seg, 2, ok_ptr, 7, tq.UNIFORM, 0, 0, ok_ptr, need, None) == tq.ERR_INVALID_ARG
